@@ -1,0 +1,219 @@
+"""CPU oracle for the Strassen-Winograd hot path -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline legs may import
+this package; the product library never does, and this package never imports the
+product.  It wraps ``strassen_oracle.c`` (plain C, FP64, compiled here with gcc,
+``-O2 -ffp-contract=off -fopenmp``) and adds the host-side arithmetic of the
+paper that needs no matrix data:
+
+* ``classical`` / ``classical_samples`` -- the definition C = A.B (Algorithm 1,
+  "Ensure C = A.B"), k ascending, multiply and add never fused.
+* ``strassen_winograd`` -- the sequential Strassen-Winograd recursion of
+  Appendix A (typos of the printed table corrected), cutoff to classical
+  (Section 5.4), dynamic peeling for odd sizes (Section 3.1), per-level 'B'
+  (U-chain combine) or 'D' (one Q at a time folded into C, Algorithm 1).
+* ``level_sizes``, ``flops_recurrence``, ``flops_closed_form`` -- the cost
+  F(n) = c_s n^{log2 7} - 5 n^2, c_s = (2 n0 + 4) / n0^{log2 7 - 2} (Appendix A).
+* ``workspace_words`` -- the memory recurrences of Sections 3.3.1 and 3.4.1
+  (a BFS step stores 7 triples S_j,T_j,Q_j of quarter size, a DFS step one),
+  ``mem_um_closed_form`` -- Mem_UM = 7 n^2 / P^{2/w0} - 4 n^2 / P at P = 7^k.
+* ``effective_gflops`` -- 2 n^3 / (t 10^9) (Section 5.2).
+
+Every function is pinned by tests/test_oracle_*.py to something other than
+itself (closed forms, a hand-worked product, brute-force equality on integer
+data, the paper's closed-form counts); none is "parity unpinned" except values at
+sizes where no full classical product can be computed, where sampled entries of
+the definition are used instead.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "strassen_oracle.c")
+_LIB = os.path.join(_HERE, "_build", "libstrassen_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+class Counters(ctypes.Structure):
+    _fields_ = [("base_calls", ctypes.c_int64), ("mults", ctypes.c_int64),
+                ("adds", ctypes.c_int64), ("block_adds", ctypes.c_int64),
+                ("peels", ctypes.c_int64)]
+
+    def as_dict(self):
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no FMA contraction, OpenMP over rows)."""
+    os.makedirs(os.path.dirname(_LIB), exist_ok=True)
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+                               "-std=c11", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            P = ctypes.c_void_p
+            I = ctypes.c_int64
+            lib.oracle_classical.argtypes = [P, I, P, I, P, I, I, I, I]
+            lib.oracle_classical.restype = None
+            lib.oracle_classical_samples.argtypes = [P, I, P, I, I, P, P, I, P]
+            lib.oracle_classical_samples.restype = None
+            lib.oracle_sw.argtypes = [P, I, P, I, P, I, I, I, ctypes.c_char_p, ctypes.POINTER(Counters)]
+            lib.oracle_sw.restype = ctypes.c_int
+            _lib = lib
+    return _lib
+
+
+def _mat(x):
+    a = np.ascontiguousarray(x, dtype=np.float64)
+    if a.ndim != 2:
+        raise ValueError("expected a 2-D array")
+    return a
+
+
+def cores() -> int:
+    """Threads the C oracle uses (OpenMP default = CPUs this process may run on)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env.split(",")[0])
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def classical(A, B):
+    """C = A.B from the definition (m x k times k x n), FP64."""
+    A, B = _mat(A), _mat(B)
+    m, k = A.shape
+    k2, n = B.shape
+    if k != k2:
+        raise ValueError("inner dimensions differ")
+    C = np.empty((m, n), dtype=np.float64)
+    _load().oracle_classical(A.ctypes.data, max(k, 1), B.ctypes.data, max(n, 1), C.ctypes.data, max(n, 1), m, n, k)
+    return C
+
+
+def classical_samples(A, B, rows, cols):
+    """Entries C[rows[t], cols[t]] of A.B from the definition."""
+    A, B = _mat(A), _mat(B)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    if rows.shape != cols.shape or A.shape[1] != B.shape[0]:
+        raise ValueError("shape mismatch")
+    if rows.size and (rows.min() < 0 or rows.max() >= A.shape[0] or cols.min() < 0 or cols.max() >= B.shape[1]):
+        raise IndexError("sample out of range")
+    out = np.empty(rows.shape, dtype=np.float64)
+    _load().oracle_classical_samples(A.ctypes.data, A.shape[1], B.ctypes.data, B.shape[1], A.shape[1],
+                                     rows.ctypes.data, cols.ctypes.data, rows.size, out.ctypes.data)
+    return out
+
+
+def strassen_winograd(A, B, cutoff, schedule=None):
+    """(C, counters) with C = A.B by Strassen-Winograd, recursing while size > cutoff."""
+    A, B = _mat(A), _mat(B)
+    n = A.shape[0]
+    if A.shape != (n, n) or B.shape != (n, n):
+        raise ValueError("square matrices of equal size expected")
+    C = np.empty((n, n), dtype=np.float64)
+    cnt = Counters()
+    sched = None if schedule is None else schedule.encode()
+    rc = _load().oracle_sw(A.ctypes.data, n, B.ctypes.data, n, C.ctypes.data, n, n, int(cutoff), sched,
+                           ctypes.byref(cnt))
+    if rc != 0:
+        raise RuntimeError("oracle_sw failed with status %d" % rc)
+    return C, cnt.as_dict()
+
+
+# ---------------------------------------------------------------------------
+# host-side arithmetic of the paper (no matrix data)
+# ---------------------------------------------------------------------------
+
+def level_sizes(n: int, cutoff: int):
+    """[m_0 = n, m_1, ..., m_L]: halve (dropping a peeled row/column) while m > cutoff."""
+    if n < 1 or cutoff < 1:
+        raise ValueError("n and cutoff must be positive")
+    m = [n]
+    while m[-1] > cutoff:
+        m.append(m[-1] // 2)
+    return m
+
+
+def flops_recurrence(n: int, cutoff: int) -> int:
+    """Flops of Strassen-Winograd for n = n0 2^L (no odd size on the way):
+    7^L classical products of 2 n0^3 - n0^2 flops plus 15 quadrant additions per node."""
+    m = level_sizes(n, cutoff)
+    L = len(m) - 1
+    if any(x % 2 for x in m[:-1]):
+        raise ValueError("closed form holds only when no level is peeled")
+    n0 = m[-1]
+    return 7 ** L * (2 * n0 ** 3 - n0 ** 2) + 15 * sum(7 ** i * m[i + 1] ** 2 for i in range(L))
+
+
+def flops_closed_form(n: int, n0: int) -> float:
+    """F(n) = c_s n^{w0} - 5 n^2 with c_s = (2 n0 + 4) / n0^{w0 - 2}, w0 = log2 7 (Appendix A)."""
+    w0 = math.log2(7.0)
+    cs = (2 * n0 + 4) / n0 ** (w0 - 2)
+    return cs * n ** w0 - 5.0 * n * n
+
+
+def workspace_words(n: int, cutoff: int, schedule: str, batch: int = 1, accounting: int = 21) -> int:
+    """Words beyond A, B, C for a per-level schedule string (top level first).
+
+    Sections 3.3.1 / 3.4.1: a BFS step stores all 7 triples (S_j, T_j, Q_j) of quarter
+    size per parent, a DFS step one triple.  accounting=21 counts every triple in full
+    (the paper's figure); accounting=15 counts, at BFS levels, only the 4+4 operand sums
+    that are not plain quadrants plus the 7 products (15 of the 21 quarter matrices).
+    """
+    m = level_sizes(n, cutoff)
+    L = len(m) - 1
+    if len(schedule) != L or any(c not in "BD" for c in schedule):
+        raise ValueError("schedule must have one 'B' or 'D' per level (%d levels)" % L)
+    if accounting not in (15, 21):
+        raise ValueError("accounting is 21 (paper) or 15 (quadrant operands as views)")
+    words, live = 0, batch
+    for i, c in enumerate(schedule):
+        h = m[i + 1]
+        if c == "B":
+            words += live * accounting * h * h
+            live *= 7
+        else:
+            words += live * 3 * h * h
+    return words
+
+
+def mem_um_closed_form(n: int, k: int) -> float:
+    """Mem_UM(n, P = 7^k) * P = 7 n^2 (7/4)^k - 4 n^2: total words of A, B, C plus all
+    temporaries of k BFS steps, summed over the P processors (Section 3.3.1)."""
+    return 7.0 * n * n * (7.0 / 4.0) ** k - 4.0 * n * n
+
+
+def lm_schedule(n: int, cutoff: int, budget_words: int, batch: int = 1, accounting: int = 21) -> str:
+    """Limited-Memory rule (Section 3.4): the fewest leading DFS steps, followed by
+    BFS steps only, whose temporaries fit the budget."""
+    L = len(level_sizes(n, cutoff)) - 1
+    for ell in range(L + 1):
+        s = "D" * ell + "B" * (L - ell)
+        if workspace_words(n, cutoff, s, batch, accounting) <= budget_words:
+            return s
+    raise ValueError("even the all-DFS schedule does not fit the budget")
+
+
+def effective_gflops(n: int, seconds: float, batch: int = 1) -> float:
+    """Effective GFLOPS = 2 n^3 / (seconds 10^9) (Section 5.2), times the batch size."""
+    return 2.0 * n ** 3 * batch / (seconds * 1e9)
