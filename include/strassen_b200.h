@@ -1,0 +1,187 @@
+/*
+ * strassen_b200 -- C ABI of the single-GPU (NVIDIA B200, sm_100a) hot path of CAPS,
+ * the communication-avoiding parallel Strassen algorithm (Ballard, Demmel, Holtz,
+ * Lipshitz, Schwartz): the Strassen-Winograd recursion computing C = A.B for n x n
+ * FP64 matrices.
+ *
+ * What one call computes (paper passages in brackets):
+ *   - operand formation: the A-side sums T2..T5 and B-side sums S2,S3,S4,S6 of every
+ *     live node; the other six operands are plain quadrants and are used in place
+ *     [Appendix A; Algorithm 1 "locally compute the S_i's and T_i's"];
+ *   - 7^L base-case classical products Q_j = T_j.S_j, one batched FP64 GEMM launch per
+ *     group of live leaves [Section 5.4 "switches to classical below some size n0";
+ *     Algorithm 2 "localStrassen"];
+ *   - recombination of the Q_j into the four quadrants of C through U1..U3
+ *     [Appendix A; Algorithm 1 "locally compute C from all the Q_i's"];
+ *   - each recursion level runs as a BFS step (all seven sub-problems materialised and
+ *     batched) or a DFS step (one sub-problem at a time, its Q_j folded into C and
+ *     discarded) [Section 3.1; Algorithm 1], the mix chosen by the workspace budget
+ *     with the Limited-Memory rule: the fewest leading DFS steps, then BFS steps only
+ *     [Section 3.4];
+ *   - odd sizes are handled by dynamic peeling of the last row and column at every
+ *     level whose size is odd [Section 3.1 names padding or dynamic peeling].
+ *
+ * Conventions for every entry point:
+ *   - matrices are row-major FP64; "device pointer" means memory the GPU can address
+ *     (cudaMalloc or equivalent), "host pointer" ordinary (preferably pinned) host memory;
+ *   - functions returning int return STRASSEN_OK (0) or a negative strassen_status;
+ *     functions returning a pointer return NULL on failure; either way a description of
+ *     the failure is available from strassen_last_error() on the calling thread;
+ *   - the library never aborts, throws, or traps on the device; there is no CPU
+ *     fallback: without a usable CUDA device the compute calls fail with
+ *     STRASSEN_CUDA_ERROR.
+ */
+#ifndef STRASSEN_B200_H
+#define STRASSEN_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct strassen_plan strassen_plan; /* opaque host object */
+
+typedef enum strassen_status {
+    STRASSEN_OK = 0,
+    STRASSEN_INVALID_ARG = -1,         /* NULL pointer, n < 1, cutoff < 1, batch < 1, ld < n ...       */
+    STRASSEN_BAD_SCHEDULE = -2,        /* wrong length or a character other than 'B' / 'D'            */
+    STRASSEN_WORKSPACE_TOO_SMALL = -3, /* supplied workspace or budget smaller than the plan needs    */
+    STRASSEN_ALIAS = -4,               /* C overlaps A or B                                           */
+    STRASSEN_MISALIGNED = -5,          /* a matrix or workspace pointer is not 8-byte (256-byte) aligned */
+    STRASSEN_CUDA_ERROR = -6,          /* a CUDA runtime call failed; text in strassen_last_error()   */
+    STRASSEN_OUT_OF_MEMORY = -7        /* host or device allocation failed                            */
+} strassen_status;
+
+/* Kernel families, used as indices by strassen_plan_get_timings / strassen_plan_launches_of. */
+typedef enum strassen_kernel_kind {
+    STRASSEN_K_FORM = 0,       /* BFS operand formation: T2..T5, S2,S3,S4,S6 of every parent       */
+    STRASSEN_K_GEMM = 1,       /* batched base-case products                                        */
+    STRASSEN_K_RECOMBINE = 2,  /* BFS recombination: U-chain, four quadrants of C                   */
+    STRASSEN_K_FORM_ONE = 3,   /* DFS operand formation of one sub-problem j                        */
+    STRASSEN_K_ACCUMULATE = 4, /* DFS fold of one Q_j into the quadrants of C                       */
+    STRASSEN_K_PEEL = 5,       /* peeling fix-ups: rank-one update, last column, last row           */
+    STRASSEN_K_COUNT = 6
+} strassen_kernel_kind;
+
+/* Extended plan description.  Zero-initialise, then set what differs from the default. */
+typedef struct strassen_options {
+    int64_t n;              /* matrix size, >= 1                                                   */
+    int64_t cutoff;         /* recurse while the current size is > cutoff; >= 1                    */
+    const char *schedule;   /* one 'B' or 'D' per level, top level first; NULL or "auto" = LM rule */
+    int64_t batch;          /* independent products per call; 0 means 1                            */
+    int64_t lda, ldb, ldc;  /* leading dimensions in elements; 0 means n                           */
+    int64_t stride_a, stride_b, stride_c; /* element distance between batch members; 0 means ld * n */
+    size_t workspace_budget_bytes;  /* for "auto": largest workspace allowed; 0 = free device memory
+                                       of the current device minus a 1 GiB margin                  */
+} strassen_options;
+
+/*
+ * strassen_plan_create -- plan C = A.B for n x n matrices [Algorithm 1 "Require A, B n x n"].
+ *   n        matrix size (>= 1), contiguous rows (ld = n), one product per call.
+ *   cutoff   base-case size n0 (>= 1): a node of size m is split while m > cutoff, so the
+ *            level sizes are m_0 = n, m_{i+1} = floor(m_i / 2); n <= cutoff gives zero
+ *            levels, i.e. one classical product [Section 5.4].
+ *   schedule host string, one character per level from the top: 'B' = BFS step, 'D' = DFS
+ *            step [Section 3.1].  NULL or "auto" applies the Limited-Memory rule
+ *            [Section 3.4] against the free memory of the current device.
+ * Host-only: no device memory is touched until the first strassen_dgemm.  The string is
+ * copied.  Returns NULL on failure (see strassen_last_error).
+ */
+strassen_plan *strassen_plan_create(int64_t n, int64_t cutoff, const char *schedule);
+
+/* strassen_plan_create_ex -- as above with batch, leading dimensions, batch strides and an
+ * explicit workspace budget.  `opt` and the string it points to are host memory, read only
+ * during the call. */
+strassen_plan *strassen_plan_create_ex(const strassen_options *opt);
+
+/*
+ * strassen_dgemm -- enqueue C = A.B on `stream` [Algorithm 1; Appendix A].
+ *   A, B   device pointers, row-major, n rows of lda / ldb elements (batch members stride_a /
+ *          stride_b apart); read only, never written.
+ *   C      device pointer, same layout with ldc / stride_c; fully overwritten.  C must not
+ *          overlap A or B (checked by address range -> STRASSEN_ALIAS).
+ *   stream a cudaStream_t passed as void* (NULL = the legacy default stream).
+ * All pointers must be 8-byte aligned (STRASSEN_MISALIGNED otherwise); 16-byte alignment
+ * with even leading dimensions selects the vectorised paths.  Asynchronous: returns once
+ * the kernels are enqueued; no host synchronisation inside, except on the first call of
+ * a plan, which uploads the plan's node tables and, unless strassen_plan_set_workspace was
+ * called, allocates the workspace (cudaMalloc) -- make that first call outside any stream
+ * capture.  One call per plan may be in flight at a time (the workspace is shared).
+ * The caller owns A, B, C.  NaN / Inf inputs give unspecified results (the operand sums
+ * can turn Inf into NaN where the classical product would not).
+ */
+int strassen_dgemm(strassen_plan *plan, const double *A, const double *B, double *C, void *stream);
+
+/*
+ * strassen_dgemm_host -- the same product for HOST matrices: copies A and B to device
+ * staging buffers owned by the plan (allocated on first use), runs strassen_dgemm and
+ * copies C back, all enqueued on `stream`; the host buffers must stay valid until the
+ * stream has been synchronised.  Host rows are contiguous (ld = n) and batch members n*n
+ * apart.  Pinned host memory makes the copies asynchronous.
+ */
+int strassen_dgemm_host(strassen_plan *plan, const double *hostA, const double *hostB, double *hostC,
+                        void *stream);
+
+/* strassen_plan_destroy -- free the plan, its device tables, staging buffers and any
+ * workspace it allocated itself (not one given by strassen_plan_set_workspace).  The caller
+ * must have synchronised the streams the plan was used on.  NULL is ignored. */
+void strassen_plan_destroy(strassen_plan *plan);
+
+/* Bytes of device workspace the resolved schedule needs beyond A, B, C: per BFS level the
+ * 4 + 4 operand sums and 7 products of every parent, per DFS level one (T, S, Q) triple per
+ * parent, rows padded to a multiple of 4 elements [Sections 3.3.1, 3.4.1: a BFS step stores
+ * 7 triples, a DFS step one; the six quadrant operands are used in place here]. */
+size_t strassen_plan_workspace_bytes(const strassen_plan *plan);
+
+/* Give the plan caller-owned device memory to use as workspace (256-byte aligned, at least
+ * strassen_plan_workspace_bytes).  The plan never frees it.  May be called again between
+ * products. */
+int strassen_plan_set_workspace(strassen_plan *plan, void *device_ptr, size_t bytes);
+
+/* The resolved schedule string ('B'/'D' per level; "" when there are zero levels).  Owned by
+ * the plan. */
+const char *strassen_plan_schedule(const strassen_plan *plan);
+
+int strassen_plan_levels(const strassen_plan *plan);                    /* L                         */
+int64_t strassen_plan_level_size(const strassen_plan *plan, int level); /* m_level, 0 <= level <= L  */
+int64_t strassen_plan_base_size(const strassen_plan *plan);             /* m_L                        */
+int64_t strassen_plan_base_products(const strassen_plan *plan);         /* batch * 7^L                */
+int64_t strassen_plan_launch_count(const strassen_plan *plan);          /* kernels per strassen_dgemm */
+int64_t strassen_plan_launches_of(const strassen_plan *plan, int kind); /* ... of one family          */
+
+/* Workspace (bytes, unpadded) a schedule string needs under the paper's accounting of 21
+ * quarter-size matrices per BFS parent and 3 per DFS parent [Sections 3.3.1, 3.4.1], or,
+ * with accounting = 15, counting the six quadrant operands of a BFS step as views.
+ * Returns 0 and sets the error text if the arguments are invalid. */
+size_t strassen_schedule_model_bytes(int64_t n, int64_t cutoff, int64_t batch, const char *schedule,
+                                     int accounting);
+
+/*
+ * Per-family device timing [Section 5.2: the paper times the whole product; the split is an
+ * addition for roofline reporting].  With timing enabled every launch is bracketed by CUDA
+ * events on the call's stream; strassen_plan_get_timings synchronises those events and adds
+ * their durations into ms_out[STRASSEN_K_COUNT] (milliseconds since timing was enabled or
+ * last read), then clears them.  Off by default.
+ */
+int strassen_plan_set_timing(strassen_plan *plan, int enabled);
+int strassen_plan_get_timings(strassen_plan *plan, double *ms_out /* [STRASSEN_K_COUNT] */);
+
+/*
+ * strassen_probe_fp64 -- measure the FP64 arithmetic rate of the current device with a
+ * register-resident loop (no memory traffic): kind 0 = scalar fused multiply-add, kind 1..4 =
+ * the FP64 tensor-core instruction mma.sync m8n8k4 / m16n8k4 / m16n8k8 / m16n8k16.  Runs
+ * `iters` inner iterations per thread on every SM, synchronises, and writes the achieved
+ * TFLOP/s to *tflops_out (host pointer).  Measurement aid for the roofline denominator; the
+ * paper has no counterpart.
+ */
+int strassen_probe_fp64(int kind, int64_t iters, void *stream, double *tflops_out);
+
+/* Text describing the last failure on the calling thread ("" if none).  Thread-local. */
+const char *strassen_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STRASSEN_B200_H */

@@ -1,1 +1,127 @@
-"""B200-native Strassen-Winograd (CAPS single-GPU hot path)."""
+"""B200-native Strassen-Winograd product C = A.B (the single-GPU hot path of CAPS).
+
+The work is done by ``libstrassen_b200.so`` (CUDA, sm_100a; C ABI in
+``include/strassen_b200.h``).  ``binding`` mirrors that ABI one to one; ``Plan`` adds
+only what PyTorch is used for here: device memory for C and the workspace, and the
+current CUDA stream.  Nothing in this package computes on the CPU.
+"""
+from __future__ import annotations
+
+from . import binding
+from .binding import StrassenError  # noqa: F401
+
+__all__ = ["Plan", "matmul", "binding", "StrassenError"]
+
+
+class Plan:
+    """A planned product for n x n FP64 matrices (optionally a batch of them).
+
+    ``schedule`` is one 'B' (breadth-first step) or 'D' (depth-first step) per recursion
+    level, or None / "auto" for the Limited-Memory rule against ``workspace_budget_bytes``.
+    """
+
+    def __init__(self, n, cutoff, schedule=None, batch=1, workspace_budget_bytes=0, lda=0, ldb=0, ldc=0,
+                 stride_a=0, stride_b=0, stride_c=0):
+        self.n, self.cutoff, self.batch = int(n), int(cutoff), int(batch)
+        self._h = binding.strassen_plan_create_ex(n, cutoff, schedule, batch, lda, ldb, ldc, stride_a, stride_b,
+                                                  stride_c, workspace_budget_bytes)
+        self._ws = None
+
+    # -- introspection -------------------------------------------------------------
+    @property
+    def handle(self):
+        return self._h
+
+    @property
+    def schedule(self):
+        return binding.strassen_plan_schedule(self._h)
+
+    @property
+    def levels(self):
+        return binding.strassen_plan_levels(self._h)
+
+    @property
+    def level_sizes(self):
+        return [binding.strassen_plan_level_size(self._h, i) for i in range(self.levels + 1)]
+
+    @property
+    def base_size(self):
+        return binding.strassen_plan_base_size(self._h)
+
+    @property
+    def base_products(self):
+        return binding.strassen_plan_base_products(self._h)
+
+    @property
+    def workspace_bytes(self):
+        return binding.strassen_plan_workspace_bytes(self._h)
+
+    @property
+    def launch_count(self):
+        return binding.strassen_plan_launch_count(self._h)
+
+    def launches_by_kind(self):
+        return {k: binding.strassen_plan_launches_of(self._h, i) for i, k in enumerate(binding.KERNEL_KINDS)}
+
+    # -- execution -----------------------------------------------------------------
+    def _ensure_workspace(self, device):
+        import torch
+        need = self.workspace_bytes
+        if need and self._ws is None:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=device)
+            binding.strassen_plan_set_workspace(self._h, self._ws.data_ptr(), need)
+
+    def __call__(self, A, B, out=None):
+        """C = A @ B for CUDA float64 tensors, enqueued on the current stream."""
+        import torch
+        if not (A.is_cuda and B.is_cuda and A.dtype == torch.float64 and B.dtype == torch.float64):
+            raise ValueError("A and B must be CUDA float64 tensors (there is no CPU path)")
+        if not (A.is_contiguous() and B.is_contiguous()):
+            raise ValueError("A and B must be contiguous")
+        if out is None:
+            out = torch.empty_like(A)
+        self._ensure_workspace(A.device)
+        with torch.cuda.device(A.device):
+            stream = torch.cuda.current_stream().cuda_stream
+            binding.strassen_dgemm(self._h, A.data_ptr(), B.data_ptr(), out.data_ptr(), stream)
+        return out
+
+    def run_host(self, A, B, out):
+        """The same product for host (ideally pinned) tensors, copies included, on the current stream."""
+        import torch
+        self._ensure_workspace(torch.device("cuda", torch.cuda.current_device()))
+        stream = torch.cuda.current_stream().cuda_stream
+        binding.strassen_dgemm_host(self._h, A.data_ptr(), B.data_ptr(), out.data_ptr(), stream)
+        return out
+
+    def set_timing(self, enabled=True):
+        binding.strassen_plan_set_timing(self._h, enabled)
+
+    def timings_ms(self):
+        return binding.strassen_plan_get_timings(self._h)
+
+    def close(self):
+        if self._h:
+            binding.strassen_plan_destroy(self._h)
+            self._h = None
+            self._ws = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def matmul(A, B, cutoff=512, schedule=None, workspace_budget_bytes=0):
+    """One-shot C = A @ B for square CUDA float64 tensors (2-D, or 3-D for a batch)."""
+    import torch
+    batch = 1 if A.dim() == 2 else A.shape[0]
+    n = A.shape[-1]
+    plan = Plan(n, cutoff, schedule, batch=batch, workspace_budget_bytes=workspace_budget_bytes)
+    try:
+        C = plan(A, B)
+        torch.cuda.current_stream().synchronize()
+    finally:
+        plan.close()
+    return C

@@ -1,0 +1,179 @@
+"""Thin ctypes binding of libstrassen_b200.so -- argument marshalling only.
+
+Every function here has the name of the C entry point it calls (include/strassen_b200.h)
+and does no arithmetic of the method: all steps run in the library's CUDA kernels.
+There is no fallback: if the shared library has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstrassen_b200.so")
+
+STRASSEN_OK = 0
+STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SCHEDULE", -3: "WORKSPACE_TOO_SMALL", -4: "ALIAS",
+                -5: "MISALIGNED", -6: "CUDA_ERROR", -7: "OUT_OF_MEMORY"}
+K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_COUNT = range(7)
+KERNEL_KINDS = ("form", "gemm", "recombine", "form_one", "accumulate", "peel")
+
+# every symbol the header declares: (name, restype, argtypes)
+_vp, _i64, _sz, _cp, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_char_p, ctypes.c_int
+_dp = ctypes.POINTER(ctypes.c_double)
+
+
+class strassen_options(ctypes.Structure):
+    _fields_ = [("n", _i64), ("cutoff", _i64), ("schedule", _cp), ("batch", _i64),
+                ("lda", _i64), ("ldb", _i64), ("ldc", _i64),
+                ("stride_a", _i64), ("stride_b", _i64), ("stride_c", _i64),
+                ("workspace_budget_bytes", _sz)]
+
+
+SYMBOLS = [
+    ("strassen_plan_create", _vp, [_i64, _i64, _cp]),
+    ("strassen_plan_create_ex", _vp, [ctypes.POINTER(strassen_options)]),
+    ("strassen_dgemm", _int, [_vp, _vp, _vp, _vp, _vp]),
+    ("strassen_dgemm_host", _int, [_vp, _vp, _vp, _vp, _vp]),
+    ("strassen_plan_destroy", None, [_vp]),
+    ("strassen_plan_workspace_bytes", _sz, [_vp]),
+    ("strassen_plan_set_workspace", _int, [_vp, _vp, _sz]),
+    ("strassen_plan_schedule", _cp, [_vp]),
+    ("strassen_plan_levels", _int, [_vp]),
+    ("strassen_plan_level_size", _i64, [_vp, _int]),
+    ("strassen_plan_base_size", _i64, [_vp]),
+    ("strassen_plan_base_products", _i64, [_vp]),
+    ("strassen_plan_launch_count", _i64, [_vp]),
+    ("strassen_plan_launches_of", _i64, [_vp, _int]),
+    ("strassen_schedule_model_bytes", _sz, [_i64, _i64, _i64, _cp, _int]),
+    ("strassen_plan_set_timing", _int, [_vp, _int]),
+    ("strassen_plan_get_timings", _int, [_vp, _dp]),
+    ("strassen_probe_fp64", _int, [_int, _i64, _vp, _dp]),
+    ("strassen_last_error", _cp, []),
+]
+
+_lib = None
+
+
+class StrassenError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("%s (%d): %s" % (STATUS_NAMES.get(status, "?"), status, message))
+        self.status = status
+
+
+def lib() -> ctypes.CDLL:
+    """Load the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libstrassen_b200.so is missing: run `python -m paper_1202_3173_b200.build` "
+                               "(there is no fallback path)")
+        l = ctypes.CDLL(LIB_PATH)
+        for name, res, args in SYMBOLS:
+            f = getattr(l, name)
+            f.restype, f.argtypes = res, args
+        _lib = l
+    return _lib
+
+
+def strassen_last_error() -> str:
+    return lib().strassen_last_error().decode()
+
+
+def _check(status: int) -> None:
+    if status != STRASSEN_OK:
+        raise StrassenError(status, strassen_last_error())
+
+
+def _sched(schedule):
+    return None if schedule is None else schedule.encode()
+
+
+def strassen_plan_create(n: int, cutoff: int, schedule) -> int:
+    h = lib().strassen_plan_create(n, cutoff, _sched(schedule))
+    if not h:
+        raise StrassenError(-1, strassen_last_error())
+    return h
+
+
+def strassen_plan_create_ex(n, cutoff, schedule=None, batch=1, lda=0, ldb=0, ldc=0, stride_a=0, stride_b=0,
+                            stride_c=0, workspace_budget_bytes=0) -> int:
+    o = strassen_options(n, cutoff, _sched(schedule), batch, lda, ldb, ldc, stride_a, stride_b, stride_c,
+                         workspace_budget_bytes)
+    h = lib().strassen_plan_create_ex(ctypes.byref(o))
+    if not h:
+        raise StrassenError(-1, strassen_last_error())
+    return h
+
+
+def strassen_dgemm(plan: int, A: int, B: int, C: int, stream: int = 0) -> None:
+    """A, B, C: device addresses (ints); stream: a cudaStream_t handle (int)."""
+    _check(lib().strassen_dgemm(plan, A, B, C, stream))
+
+
+def strassen_dgemm_host(plan: int, A: int, B: int, C: int, stream: int = 0) -> None:
+    """A, B, C: host addresses (ints)."""
+    _check(lib().strassen_dgemm_host(plan, A, B, C, stream))
+
+
+def strassen_plan_destroy(plan: int) -> None:
+    lib().strassen_plan_destroy(plan)
+
+
+def strassen_plan_workspace_bytes(plan: int) -> int:
+    return lib().strassen_plan_workspace_bytes(plan)
+
+
+def strassen_plan_set_workspace(plan: int, device_ptr: int, nbytes: int) -> None:
+    _check(lib().strassen_plan_set_workspace(plan, device_ptr, nbytes))
+
+
+def strassen_plan_schedule(plan: int) -> str:
+    return lib().strassen_plan_schedule(plan).decode()
+
+
+def strassen_plan_levels(plan: int) -> int:
+    return lib().strassen_plan_levels(plan)
+
+
+def strassen_plan_level_size(plan: int, level: int) -> int:
+    return lib().strassen_plan_level_size(plan, level)
+
+
+def strassen_plan_base_size(plan: int) -> int:
+    return lib().strassen_plan_base_size(plan)
+
+
+def strassen_plan_base_products(plan: int) -> int:
+    return lib().strassen_plan_base_products(plan)
+
+
+def strassen_plan_launch_count(plan: int) -> int:
+    return lib().strassen_plan_launch_count(plan)
+
+
+def strassen_plan_launches_of(plan: int, kind: int) -> int:
+    return lib().strassen_plan_launches_of(plan, kind)
+
+
+def strassen_schedule_model_bytes(n, cutoff, batch, schedule, accounting=21) -> int:
+    v = lib().strassen_schedule_model_bytes(n, cutoff, batch, _sched(schedule), accounting)
+    if v == 0 and strassen_last_error():
+        raise StrassenError(-2, strassen_last_error())
+    return v
+
+
+def strassen_plan_set_timing(plan: int, enabled: bool) -> None:
+    _check(lib().strassen_plan_set_timing(plan, int(enabled)))
+
+
+def strassen_plan_get_timings(plan: int):
+    out = (ctypes.c_double * K_COUNT)()
+    _check(lib().strassen_plan_get_timings(plan, out))
+    return dict(zip(KERNEL_KINDS, list(out)))
+
+
+def strassen_probe_fp64(kind: int, iters: int, stream: int = 0) -> float:
+    out = ctypes.c_double()
+    _check(lib().strassen_probe_fp64(kind, iters, stream, ctypes.byref(out)))
+    return out.value

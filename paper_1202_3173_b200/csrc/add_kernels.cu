@@ -1,0 +1,455 @@
+// Streaming kernels of one Strassen-Winograd step (Appendix A): operand formation,
+// recombination, the one-sub-problem-at-a-time variants of a DFS step (Algorithm 1) and the
+// peeling fix-ups for odd sizes.  All are HBM-bound: every element of every quadrant is read
+// once and every output element written once per level.
+//
+// Work decomposition shared by the four add kernels: a CTA of 64 x 4 threads owns a tile of
+// 16 rows x (64 * VEC) columns of one h x h quadrant position of one (node, side) item;
+// each thread handles 4 rows (stride 4) and VEC adjacent columns, issuing all of its loads
+// before the arithmetic so that 4 x (number of input streams) requests are in flight.
+#include "kernels.h"
+
+namespace strassen {
+
+namespace {
+
+constexpr int TX = 64, TY = 4, ROWS_PER_THREAD = 4, TILE_ROWS = TY * ROWS_PER_THREAD;
+constexpr int MAX_Z = 32768;   // items per launch (gridDim.z limit is 65535)
+
+template <int VEC> struct Vec;
+template <> struct Vec<1> {
+    using type = double;
+    static __device__ __forceinline__ double ld(const double *p) { return __ldcs(p); }
+    static __device__ __forceinline__ double ldk(const double *p) { return *p; }
+    static __device__ __forceinline__ void st(double *p, double v) { *p = v; }
+    static __device__ __forceinline__ double add(double a, double b) { return a + b; }
+    static __device__ __forceinline__ double sub(double a, double b) { return a - b; }
+    static __device__ __forceinline__ double neg(double a) { return -a; }
+};
+template <> struct Vec<2> {
+    using type = double2;
+    static __device__ __forceinline__ double2 ld(const double *p) { return __ldcs(reinterpret_cast<const double2 *>(p)); }
+    static __device__ __forceinline__ double2 ldk(const double *p) { return *reinterpret_cast<const double2 *>(p); }
+    static __device__ __forceinline__ void st(double *p, double2 v) { *reinterpret_cast<double2 *>(p) = v; }
+    static __device__ __forceinline__ double2 add(double2 a, double2 b) { return make_double2(a.x + b.x, a.y + b.y); }
+    static __device__ __forceinline__ double2 sub(double2 a, double2 b) { return make_double2(a.x - b.x, a.y - b.y); }
+    static __device__ __forceinline__ double2 neg(double2 a) { return make_double2(-a.x, -a.y); }
+};
+
+__device__ __forceinline__ double *resolve(const Bases &bases, const Operand &x) { return base_ptr(bases, x.base) + x.off; }
+
+// ---------------------------------------------------------------------------------------
+// BFS operand formation.  item = 2 * parent + side; side 0 forms T2..T5 from the quadrants
+// of the parent's A operand, side 1 forms S2, S3, S4, S6 from those of its B operand:
+//   T2 = A21 + A22   T3 = T2 - A11   T4 = A11 - A21   T5 = A12 - T3
+//   S2 = B12 - B11   S3 = B22 - S2   S4 = B22 - B12   S6 = S3 - B21
+// ---------------------------------------------------------------------------------------
+template <int VEC>
+__global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict__ parents,
+                                                          const Node *__restrict__ children, Bases bases, int h,
+                                                          int item0)
+{
+    using V = Vec<VEC>;
+    using T = typename V::type;
+    const int item = item0 + blockIdx.z;
+    const int par = item >> 1, side = item & 1;
+    const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
+    if (c >= h) return;
+    const Node *kids = children + size_t(par) * 7;
+    const Operand x = side ? parents[par].b : parents[par].a;
+    const double *X = resolve(bases, x);
+    const int64_t ld = x.ld;
+    const int64_t hq = int64_t(h) * ld;
+    double *o0, *o1, *o2, *o3;
+    int64_t ldo;
+    if (side == 0) {
+        o0 = resolve(bases, kids[2].a); o1 = resolve(bases, kids[3].a);
+        o2 = resolve(bases, kids[4].a); o3 = resolve(bases, kids[5].a);
+        ldo = kids[2].a.ld;
+    } else {
+        o0 = resolve(bases, kids[2].b); o1 = resolve(bases, kids[3].b);
+        o2 = resolve(bases, kids[4].b); o3 = resolve(bases, kids[6].b);
+        ldo = kids[2].b.ld;
+    }
+    const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
+    T x11[ROWS_PER_THREAD], x12[ROWS_PER_THREAD], x21[ROWS_PER_THREAD], x22[ROWS_PER_THREAD];
+#pragma unroll
+    for (int i = 0; i < ROWS_PER_THREAD; ++i) {
+        const int r = r0 + i * TY;
+        if (r < h) {
+            const double *q = X + int64_t(r) * ld + c;
+            x11[i] = V::ld(q); x12[i] = V::ld(q + h); x21[i] = V::ld(q + hq); x22[i] = V::ld(q + hq + h);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < ROWS_PER_THREAD; ++i) {
+        const int r = r0 + i * TY;
+        if (r < h) {
+            const int64_t o = int64_t(r) * ldo + c;
+            if (side == 0) {
+                const T t2 = V::add(x21[i], x22[i]);
+                const T t3 = V::sub(t2, x11[i]);
+                V::st(o0 + o, t2); V::st(o1 + o, t3);
+                V::st(o2 + o, V::sub(x11[i], x21[i]));
+                V::st(o3 + o, V::sub(x12[i], t3));
+            } else {
+                const T s2 = V::sub(x12[i], x11[i]);
+                const T s3 = V::sub(x22[i], s2);
+                V::st(o0 + o, s2); V::st(o1 + o, s3);
+                V::st(o2 + o, V::sub(x22[i], x12[i]));
+                V::st(o3 + o, V::sub(s3, x21[i]));
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// BFS recombination.  item = parent:
+//   U1 = Q0 + Q3   U2 = U1 + Q4   U3 = U1 + Q2
+//   C11 = Q0 + Q1  C12 = U3 + Q5  C21 = U2 - Q6  C22 = U2 + Q2
+// ---------------------------------------------------------------------------------------
+template <int VEC>
+__global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__restrict__ parents,
+                                                               const Node *__restrict__ children, Bases bases,
+                                                               int h, int item0)
+{
+    using V = Vec<VEC>;
+    using T = typename V::type;
+    const int par = item0 + blockIdx.z;
+    const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
+    if (c >= h) return;
+    const Node *kids = children + size_t(par) * 7;
+    const double *Q[7];
+#pragma unroll
+    for (int j = 0; j < 7; ++j) Q[j] = resolve(bases, kids[j].c);
+    const int64_t ldq = kids[0].c.ld;
+    const Operand cc = parents[par].c;
+    double *C = resolve(bases, cc);
+    const int64_t ldc = cc.ld, hq = int64_t(h) * ldc;
+    const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
+    constexpr int RP = 2;   // rows per pass: 14 vectors in flight per thread
+#pragma unroll
+    for (int pass = 0; pass < ROWS_PER_THREAD / RP; ++pass) {
+        T q[RP][7];
+#pragma unroll
+        for (int i = 0; i < RP; ++i) {
+            const int r = r0 + (pass * RP + i) * TY;
+            if (r < h) {
+#pragma unroll
+                for (int j = 0; j < 7; ++j) q[i][j] = V::ld(Q[j] + int64_t(r) * ldq + c);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < RP; ++i) {
+            const int r = r0 + (pass * RP + i) * TY;
+            if (r < h) {
+                const T u1 = V::add(q[i][0], q[i][3]);
+                const T u2 = V::add(u1, q[i][4]);
+                const T u3 = V::add(u1, q[i][2]);
+                double *o = C + int64_t(r) * ldc + c;
+                V::st(o, V::add(q[i][0], q[i][1]));
+                V::st(o + h, V::add(u3, q[i][5]));
+                V::st(o + hq, V::sub(u2, q[i][6]));
+                V::st(o + hq + h, V::add(u2, q[i][2]));
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// DFS operand formation of sub-problem j (Algorithm 1: "locally compute S_i and T_i").
+// sides: bit 0 = the A-side operand of child j is a sum, bit 1 = the B-side one is.
+// ---------------------------------------------------------------------------------------
+template <int VEC>
+__global__ void __launch_bounds__(TX *TY) form_one_kernel(const Node *__restrict__ parents,
+                                                          const Node *__restrict__ children, Bases bases, int h,
+                                                          int j, int sides, int item0)
+{
+    using V = Vec<VEC>;
+    using T = typename V::type;
+    const int item = item0 + blockIdx.z;
+    int par, side;
+    if (sides == 3) { par = item >> 1; side = item & 1; }
+    else { par = item; side = sides == 2; }
+    const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
+    if (c >= h) return;
+    const Operand x = side ? parents[par].b : parents[par].a;
+    const Operand y = side ? children[par].b : children[par].a;
+    const double *X = resolve(bases, x);
+    double *O = resolve(bases, y);
+    const int64_t ld = x.ld, hq = int64_t(h) * ld, ldo = y.ld;
+    const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
+    const int which = side * 8 + j;
+#pragma unroll
+    for (int i = 0; i < ROWS_PER_THREAD; ++i) {
+        const int r = r0 + i * TY;
+        if (r >= h) continue;
+        const double *q = X + int64_t(r) * ld + c;
+        T v;
+        switch (which) {
+        case 2: v = V::add(V::ld(q + hq), V::ld(q + hq + h)); break;                                   // T2
+        case 3: v = V::sub(V::add(V::ld(q + hq), V::ld(q + hq + h)), V::ld(q)); break;                 // T3
+        case 4: v = V::sub(V::ld(q), V::ld(q + hq)); break;                                            // T4
+        case 5: v = V::sub(V::ld(q + h), V::sub(V::add(V::ld(q + hq), V::ld(q + hq + h)), V::ld(q))); break;  // T5
+        case 10: v = V::sub(V::ld(q + h), V::ld(q)); break;                                            // S2
+        case 11: v = V::sub(V::ld(q + hq + h), V::sub(V::ld(q + h), V::ld(q))); break;                 // S3
+        case 12: v = V::sub(V::ld(q + hq + h), V::ld(q + h)); break;                                   // S4
+        default: v = V::sub(V::sub(V::ld(q + hq + h), V::sub(V::ld(q + h), V::ld(q))), V::ld(q + hq)); break;  // S6
+        }
+        V::st(O + int64_t(r) * ldo + c, v);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// DFS fold of Q_j into C (Algorithm 1: "locally compute contribution of Q_i to C"), the flat
+// form of the U chain:  C11 = Q0+Q1, C12 = Q0+Q3+Q2+Q5, C21 = Q0+Q3+Q4-Q6, C22 = Q0+Q3+Q4+Q2.
+// Q0 writes all four quadrants (first touch), later Q_j read-modify-write theirs.
+// ---------------------------------------------------------------------------------------
+template <int VEC>
+__global__ void __launch_bounds__(TX *TY) accumulate_kernel(const Node *__restrict__ parents,
+                                                            const Node *__restrict__ children, Bases bases, int h,
+                                                            int j, int item0)
+{
+    using V = Vec<VEC>;
+    using T = typename V::type;
+    const int par = item0 + blockIdx.z;
+    const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
+    if (c >= h) return;
+    const Operand qq = children[par].c, cc = parents[par].c;
+    const double *Q = resolve(bases, qq);
+    double *C = resolve(bases, cc);
+    const int64_t ldq = qq.ld, ldc = cc.ld, hq = int64_t(h) * ldc;
+    const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
+#pragma unroll
+    for (int i = 0; i < ROWS_PER_THREAD; ++i) {
+        const int r = r0 + i * TY;
+        if (r >= h) continue;
+        const T q = V::ld(Q + int64_t(r) * ldq + c);
+        double *o = C + int64_t(r) * ldc + c;
+        double *c11 = o, *c12 = o + h, *c21 = o + hq, *c22 = o + hq + h;
+        switch (j) {
+        case 0: V::st(c11, q); V::st(c12, q); V::st(c21, q); V::st(c22, q); break;
+        case 1: V::st(c11, V::add(V::ldk(c11), q)); break;
+        case 2: V::st(c12, V::add(V::ldk(c12), q)); V::st(c22, V::add(V::ldk(c22), q)); break;
+        case 3: V::st(c12, V::add(V::ldk(c12), q)); V::st(c21, V::add(V::ldk(c21), q));
+                V::st(c22, V::add(V::ldk(c22), q)); break;
+        case 4: V::st(c21, V::add(V::ldk(c21), q)); V::st(c22, V::add(V::ldk(c22), q)); break;
+        case 5: V::st(c12, V::add(V::ldk(c12), q)); break;
+        default: V::st(c21, V::sub(V::ldk(c21), q)); break;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Peeling fix-ups for an odd node size m = e + 1 (block algebra on the split
+// A = [A1 ac; ar al], B = [B1 bc; br be]):  the recursion has produced A1.B1 in C[0:e,0:e].
+//   rank-one:    C[r][c] += A[r][e] * B[e][c]            r, c < e
+//   last column: C[r][e]  = sum_k A[r][k] * B[k][e]      r < m
+//   last row:    C[e][c]  = sum_k A[e][k] * B[k][c]      c < e
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) peel_rank1_kernel(const Node *__restrict__ nodes, Bases bases, int e, int item0)
+{
+    const Node nd = nodes[item0 + blockIdx.z];
+    const int c = blockIdx.x * 64 + threadIdx.x;
+    if (c >= e) return;
+    const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
+    double *C = resolve(bases, nd.c);
+    const double b = B[int64_t(e) * nd.b.ld + c];
+    const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
+#pragma unroll
+    for (int i = 0; i < ROWS_PER_THREAD; ++i) {
+        const int r = r0 + i * TY;
+        if (r < e) {
+            double *o = C + int64_t(r) * nd.c.ld + c;
+            *o = fma(A[int64_t(r) * nd.a.ld + e], b, *o);
+        }
+    }
+}
+
+constexpr int PC_ROWS = 32, PC_CHUNK = 1024;
+__global__ void __launch_bounds__(256) peel_col_kernel(const Node *__restrict__ nodes, Bases bases, int m, int item0)
+{
+    __shared__ double bcol[PC_CHUNK];
+    const Node nd = nodes[item0 + blockIdx.y];
+    const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
+    double *C = resolve(bases, nd.c);
+    const int e = m - 1, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rbase = blockIdx.x * PC_ROWS + warp * 4;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int k0 = 0; k0 < m; k0 += PC_CHUNK) {
+        const int kn = min(PC_CHUNK, m - k0);
+        __syncthreads();
+        for (int k = threadIdx.x; k < kn; k += 256) bcol[k] = B[int64_t(k0 + k) * nd.b.ld + e];
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = rbase + i;
+            if (r < m) {
+                const double *a = A + int64_t(r) * nd.a.ld + k0;
+                double s = acc[i];
+                for (int k = lane; k < kn; k += 32) s = fma(a[k], bcol[k], s);
+                acc[i] = s;
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        double s = acc[i];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+        const int r = rbase + i;
+        if (lane == 0 && r < m) C[int64_t(r) * nd.c.ld + e] = s;
+    }
+}
+
+constexpr int PR_COLS = 32, PR_SLICES = 16;
+__global__ void __launch_bounds__(PR_COLS *PR_SLICES) peel_row_kernel(const Node *__restrict__ nodes, Bases bases,
+                                                                      int m, int item0)
+{
+    __shared__ double part[PR_SLICES][PR_COLS + 1];
+    const Node nd = nodes[item0 + blockIdx.y];
+    const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
+    double *C = resolve(bases, nd.c);
+    const int e = m - 1;
+    const int c = blockIdx.x * PR_COLS + threadIdx.x;
+    const double *arow = A + int64_t(e) * nd.a.ld;
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    if (c < e) {
+        const double *b = B + c;
+        const int64_t ldb = nd.b.ld;
+        int k = threadIdx.y;
+        for (; k + 3 * PR_SLICES < m; k += 4 * PR_SLICES) {
+            const double b0 = b[int64_t(k) * ldb], b1 = b[int64_t(k + PR_SLICES) * ldb];
+            const double b2 = b[int64_t(k + 2 * PR_SLICES) * ldb], b3 = b[int64_t(k + 3 * PR_SLICES) * ldb];
+            s0 = fma(arow[k], b0, s0);
+            s1 = fma(arow[k + PR_SLICES], b1, s1);
+            s2 = fma(arow[k + 2 * PR_SLICES], b2, s2);
+            s3 = fma(arow[k + 3 * PR_SLICES], b3, s3);
+        }
+        for (; k < m; k += PR_SLICES) s0 = fma(arow[k], b[int64_t(k) * ldb], s0);
+    }
+    part[threadIdx.y][threadIdx.x] = (s0 + s1) + (s2 + s3);
+    __syncthreads();
+    if (threadIdx.y == 0 && c < e) {
+        double s = 0.0;
+#pragma unroll
+        for (int i = 0; i < PR_SLICES; ++i) s += part[i][threadIdx.x];
+        C[int64_t(e) * nd.c.ld + c] = s;
+    }
+}
+
+dim3 tile_grid(int64_t h, int vec, int64_t items)
+{
+    return dim3(unsigned((h + TX * vec - 1) / (TX * vec)), unsigned((h + TILE_ROWS - 1) / TILE_ROWS), unsigned(items));
+}
+
+int chunks(int64_t items) { return int((items + MAX_Z - 1) / MAX_Z); }
+
+}  // namespace
+
+int launches_of(const Launch &op)
+{
+    switch (op.kind) {
+    case OP_FORM: return chunks(op.count * 2);
+    case OP_RECOMBINE: return chunks(op.count);
+    case OP_FORM_ONE: return chunks(op.count * ((op.j >= 2 && op.j <= 4) ? 2 : 1));
+    case OP_ACCUMULATE: return chunks(op.count);
+    case OP_PEEL: return 3 * chunks(op.count);
+    case OP_GEMM: return 1;
+    }
+    return 0;
+}
+
+#define FOR_CHUNKS(total)                                              \
+    for (int64_t item0 = 0, zn; item0 < (total); item0 += MAX_Z)       \
+        if ((zn = ((total) - item0 < MAX_Z ? (total) - item0 : MAX_Z)), true)
+
+cudaError_t launch_form(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
+                        int *launched)
+{
+    const dim3 block(TX, TY);
+    const int64_t total = op.count * 2;
+    FOR_CHUNKS(total) {
+        if (vec)
+            form_bfs_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
+                                                                            bases, int(op.h), int(item0));
+        else
+            form_bfs_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
+                                                                            bases, int(op.h), int(item0));
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
+                             int *launched)
+{
+    const dim3 block(TX, TY);
+    const int64_t total = op.count;
+    FOR_CHUNKS(total) {
+        if (vec)
+            recombine_bfs_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(
+                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), int(item0));
+        else
+            recombine_bfs_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(
+                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), int(item0));
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_form_one(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
+                            int *launched)
+{
+    const dim3 block(TX, TY);
+    const int j = op.j;
+    const int sides = (j >= 2 && j <= 5 ? 1 : 0) | ((j >= 2 && j <= 4) || j == 6 ? 2 : 0);
+    if (sides == 0) return cudaSuccess;
+    const int64_t total = op.count * (sides == 3 ? 2 : 1);
+    FOR_CHUNKS(total) {
+        if (vec)
+            form_one_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
+                                                                            bases, int(op.h), j, sides, int(item0));
+        else
+            form_one_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
+                                                                            bases, int(op.h), j, sides, int(item0));
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accumulate(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
+                              int *launched)
+{
+    const dim3 block(TX, TY);
+    const int64_t total = op.count;
+    FOR_CHUNKS(total) {
+        if (vec)
+            accumulate_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(
+                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), op.j, int(item0));
+        else
+            accumulate_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(
+                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), op.j, int(item0));
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_peel(const Node *tab, const Launch &op, const Bases &bases, cudaStream_t stream, int *launched)
+{
+    const int m = int(op.m), e = m - 1;
+    const int64_t total = op.count;
+    FOR_CHUNKS(total) {
+        const Node *nodes = tab + op.parent_tab;
+        peel_rank1_kernel<<<dim3((e + 63) / 64, (e + TILE_ROWS - 1) / TILE_ROWS, unsigned(zn)), dim3(64, TY), 0,
+                            stream>>>(nodes, bases, e, int(item0));
+        peel_col_kernel<<<dim3((m + PC_ROWS - 1) / PC_ROWS, unsigned(zn)), 256, 0, stream>>>(nodes, bases, m,
+                                                                                             int(item0));
+        peel_row_kernel<<<dim3((e + PR_COLS - 1) / PR_COLS, unsigned(zn)), dim3(PR_COLS, PR_SLICES), 0, stream>>>(
+            nodes, bases, m, int(item0));
+        *launched += 3;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace strassen

@@ -1,0 +1,443 @@
+// C ABI of the library (declared in include/strassen_b200.h): argument checking, lazy device
+// set-up, and replay of a plan's launch list on the caller's stream.
+#include "strassen_b200.h"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "kernels.h"
+#include "plan.h"
+
+using namespace strassen;
+
+namespace {
+
+thread_local std::string g_error;
+
+int fail(int status, const std::string &msg)
+{
+    g_error = msg;
+    return status;
+}
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    return fail(STRASSEN_CUDA_ERROR, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+struct TimedLaunch {
+    int kind;
+    cudaEvent_t start, stop;
+};
+
+}  // namespace
+
+struct strassen_plan {
+    PlanDesc d;
+    int device = -1;
+    int sm_count = 0;
+    Node *d_tab = nullptr;
+    double *ws = nullptr;
+    size_t ws_bytes = 0;
+    bool own_ws = false;
+    double *stage_a = nullptr, *stage_b = nullptr, *stage_c = nullptr;
+    bool timing = false;
+    std::vector<TimedLaunch> pending;
+    std::vector<cudaEvent_t> free_events;
+    double acc_ms[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0};
+    int64_t launches[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0};
+    int64_t launch_total = 0;
+};
+
+namespace {
+
+int64_t extent_words(int64_t n, int64_t ld, int64_t stride, int64_t batch)
+{
+    return (batch - 1) * stride + (n - 1) * ld + n;
+}
+
+bool overlap(const double *x, int64_t xw, const double *y, int64_t yw)
+{
+    const uintptr_t x0 = reinterpret_cast<uintptr_t>(x), x1 = x0 + uintptr_t(xw) * 8;
+    const uintptr_t y0 = reinterpret_cast<uintptr_t>(y), y1 = y0 + uintptr_t(yw) * 8;
+    return x0 < y1 && y0 < x1;
+}
+
+cudaEvent_t take_event(strassen_plan *p)
+{
+    if (!p->free_events.empty()) {
+        cudaEvent_t e = p->free_events.back();
+        p->free_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+// First use on a device: node tables, SM count, workspace.
+int ensure_device_state(strassen_plan *p)
+{
+    if (p->device < 0) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        if (major != 10)
+            return fail(STRASSEN_CUDA_ERROR, "this library holds sm_100a code only; the current device is not a B200-class GPU");
+        e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        p->device = dev;
+    }
+    if (!p->d_tab) {
+        const size_t bytes = p->d.nodes.size() * sizeof(Node);
+        cudaError_t e = cudaMalloc(&p->d_tab, bytes);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(node tables)");
+        e = cudaMemcpy(p->d_tab, p->d.nodes.data(), bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(node tables)");
+    }
+    const size_t need = size_t(p->d.ws_words) * 8;
+    if (need > 0 && !p->ws) {
+        cudaError_t e = cudaMalloc(&p->ws, need);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            char buf[160];
+            snprintf(buf, sizeof buf, "cudaMalloc of %zu workspace bytes failed: %s", need, cudaGetErrorString(e));
+            return fail(STRASSEN_OUT_OF_MEMORY, buf);
+        }
+        p->ws_bytes = need;
+        p->own_ws = true;
+    }
+    return STRASSEN_OK;
+}
+
+strassen_plan *create(const strassen_options &o)
+{
+    g_error.clear();
+    const int64_t n = o.n, cutoff = o.cutoff;
+    const int64_t batch = o.batch == 0 ? 1 : o.batch;
+    if (n < 1 || cutoff < 1 || batch < 1) {
+        fail(STRASSEN_INVALID_ARG, "n, cutoff and batch must be positive");
+        return nullptr;
+    }
+    if (n > (int64_t(1) << 30)) {
+        fail(STRASSEN_INVALID_ARG, "n exceeds 2^30");
+        return nullptr;
+    }
+    strassen_plan *p = new (std::nothrow) strassen_plan;
+    if (!p) {
+        fail(STRASSEN_OUT_OF_MEMORY, "out of host memory");
+        return nullptr;
+    }
+    PlanDesc &d = p->d;
+    d.n = n; d.cutoff = cutoff; d.batch = batch;
+    d.lda = o.lda ? o.lda : n; d.ldb = o.ldb ? o.ldb : n; d.ldc = o.ldc ? o.ldc : n;
+    d.stride_a = o.stride_a ? o.stride_a : d.lda * n;
+    d.stride_b = o.stride_b ? o.stride_b : d.ldb * n;
+    d.stride_c = o.stride_c ? o.stride_c : d.ldc * n;
+    const int64_t ldmax = 0x7fffffff;
+    if (d.lda < n || d.ldb < n || d.ldc < n || d.lda > ldmax || d.ldb > ldmax || d.ldc > ldmax) {
+        fail(STRASSEN_INVALID_ARG, "leading dimensions must be >= n and fit 31 bits");
+        delete p;
+        return nullptr;
+    }
+    if (d.stride_a < 0 || d.stride_b < 0 || (batch > 1 && d.stride_c < (n - 1) * d.ldc + n)) {
+        fail(STRASSEN_INVALID_ARG, "batch members of C must not overlap; strides must be non-negative");
+        delete p;
+        return nullptr;
+    }
+    d.sizes = level_sizes(n, cutoff);
+    const size_t L = d.sizes.size() - 1;
+    const bool want_auto = !o.schedule || strcmp(o.schedule, "auto") == 0;
+    if (want_auto) {
+        size_t budget = o.workspace_budget_bytes;
+        if (budget == 0 && L > 0) {
+            size_t free_b = 0, total_b = 0;
+            cudaError_t e = cudaMemGetInfo(&free_b, &total_b);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                fail(STRASSEN_CUDA_ERROR, std::string("schedule \"auto\" without a workspace budget needs a CUDA device: ") +
+                                              cudaGetErrorString(e));
+                delete p;
+                return nullptr;
+            }
+            const size_t margin = size_t(1) << 30;
+            budget = free_b > margin ? free_b - margin : 0;
+        }
+        if (!lm_schedule(d.sizes, batch, int64_t(budget / 8), &d.schedule)) {
+            fail(STRASSEN_WORKSPACE_TOO_SMALL, "even the all-DFS schedule does not fit the workspace budget");
+            delete p;
+            return nullptr;
+        }
+    } else {
+        d.schedule = o.schedule;
+        if (d.schedule.size() != L) {
+            char buf[128];
+            snprintf(buf, sizeof buf, "schedule has %zu characters but the plan has %zu levels", d.schedule.size(), L);
+            fail(STRASSEN_BAD_SCHEDULE, buf);
+            delete p;
+            return nullptr;
+        }
+        for (char c : d.schedule)
+            if (c != 'B' && c != 'D') {
+                fail(STRASSEN_BAD_SCHEDULE, "schedule characters must be 'B' or 'D'");
+                delete p;
+                return nullptr;
+            }
+        if (o.workspace_budget_bytes &&
+            size_t(actual_workspace_words(d.sizes, d.schedule, batch)) * 8 > o.workspace_budget_bytes) {
+            fail(STRASSEN_WORKSPACE_TOO_SMALL, "the schedule needs more workspace than the budget allows");
+            delete p;
+            return nullptr;
+        }
+    }
+    const std::string err = build_plan(&d);
+    if (!err.empty()) {
+        fail(STRASSEN_INVALID_ARG, err);
+        delete p;
+        return nullptr;
+    }
+    for (const Launch &op : d.launches) {
+        const int k = launches_of(op);
+        p->launches[op.kind] += k;
+        p->launch_total += k;
+    }
+    return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+strassen_plan *strassen_plan_create(int64_t n, int64_t cutoff, const char *schedule)
+{
+    strassen_options o;
+    memset(&o, 0, sizeof o);
+    o.n = n; o.cutoff = cutoff; o.schedule = schedule;
+    return create(o);
+}
+
+strassen_plan *strassen_plan_create_ex(const strassen_options *opt)
+{
+    if (!opt) {
+        fail(STRASSEN_INVALID_ARG, "options pointer is NULL");
+        return nullptr;
+    }
+    return create(*opt);
+}
+
+int strassen_dgemm(strassen_plan *p, const double *A, const double *B, double *C, void *stream_v)
+{
+    g_error.clear();
+    if (!p || !A || !B || !C) return fail(STRASSEN_INVALID_ARG, "plan, A, B and C must be non-NULL");
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C);
+    if (bits & 7) return fail(STRASSEN_MISALIGNED, "A, B and C must be 8-byte aligned");
+    const PlanDesc &d = p->d;
+    const int64_t wa = extent_words(d.n, d.lda, d.stride_a, d.batch), wb = extent_words(d.n, d.ldb, d.stride_b, d.batch),
+                  wc = extent_words(d.n, d.ldc, d.stride_c, d.batch);
+    if (overlap(C, wc, A, wa) || overlap(C, wc, B, wb)) return fail(STRASSEN_ALIAS, "C overlaps A or B");
+    const int rc = ensure_device_state(p);
+    if (rc != STRASSEN_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    Bases bases;
+    bases.p[BASE_A] = const_cast<double *>(A);
+    bases.p[BASE_B] = const_cast<double *>(B);
+    bases.p[BASE_C] = C;
+    bases.p[BASE_WS] = p->ws;
+    const bool bases16 = ((bits | reinterpret_cast<uintptr_t>(p->ws)) & 15) == 0;
+    int launched = 0;
+    for (const Launch &op : d.launches) {
+        const bool vec = op.vec_ok && bases16;
+        TimedLaunch t{op.kind, nullptr, nullptr};
+        if (p->timing) {
+            t.start = take_event(p);
+            t.stop = take_event(p);
+            cudaEventRecord(t.start, stream);
+        }
+        cudaError_t e = cudaSuccess;
+        switch (op.kind) {
+        case OP_FORM: e = launch_form(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_GEMM: e = launch_gemm(p->d_tab, op, bases, p->sm_count, stream, &launched); break;
+        case OP_RECOMBINE: e = launch_recombine(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_FORM_ONE: e = launch_form_one(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_ACCUMULATE: e = launch_accumulate(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_PEEL: e = launch_peel(p->d_tab, op, bases, stream, &launched); break;
+        }
+        if (p->timing) {
+            cudaEventRecord(t.stop, stream);
+            p->pending.push_back(t);
+        }
+        if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    }
+    return STRASSEN_OK;
+}
+
+int strassen_dgemm_host(strassen_plan *p, const double *hA, const double *hB, double *hC, void *stream_v)
+{
+    g_error.clear();
+    if (!p || !hA || !hB || !hC) return fail(STRASSEN_INVALID_ARG, "plan, A, B and C must be non-NULL");
+    const PlanDesc &d = p->d;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t wa = size_t(extent_words(d.n, d.lda, d.stride_a, d.batch)) * 8;
+    const size_t wb = size_t(extent_words(d.n, d.ldb, d.stride_b, d.batch)) * 8;
+    const size_t wc = size_t(extent_words(d.n, d.ldc, d.stride_c, d.batch)) * 8;
+    if (!p->stage_a) {
+        cudaError_t e = cudaMalloc(&p->stage_a, wa);
+        if (e == cudaSuccess) e = cudaMalloc(&p->stage_b, wb);
+        if (e == cudaSuccess) e = cudaMalloc(&p->stage_c, wc);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(p->stage_a); cudaFree(p->stage_b); cudaFree(p->stage_c);
+            p->stage_a = p->stage_b = p->stage_c = nullptr;
+            return fail(STRASSEN_OUT_OF_MEMORY, std::string("staging buffers: ") + cudaGetErrorString(e));
+        }
+    }
+    const size_t row = size_t(d.n) * 8;
+    auto copy_in = [&](double *dst, int64_t ld, int64_t stride, const double *src) -> cudaError_t {
+        if (ld == d.n && stride == d.n * d.n)
+            return cudaMemcpyAsync(dst, src, row * size_t(d.n) * size_t(d.batch), cudaMemcpyHostToDevice, stream);
+        for (int64_t b = 0; b < d.batch; ++b) {
+            cudaError_t e = cudaMemcpy2DAsync(dst + b * stride, size_t(ld) * 8, src + b * d.n * d.n, row, row, size_t(d.n),
+                                              cudaMemcpyHostToDevice, stream);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    };
+    cudaError_t e = copy_in(p->stage_a, d.lda, d.stride_a, hA);
+    if (e == cudaSuccess) e = copy_in(p->stage_b, d.ldb, d.stride_b, hB);
+    if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
+    const int rc = strassen_dgemm(p, p->stage_a, p->stage_b, p->stage_c, stream_v);
+    if (rc != STRASSEN_OK) return rc;
+    if (d.ldc == d.n && d.stride_c == d.n * d.n) {
+        e = cudaMemcpyAsync(hC, p->stage_c, row * size_t(d.n) * size_t(d.batch), cudaMemcpyDeviceToHost, stream);
+    } else {
+        for (int64_t b = 0; b < d.batch && e == cudaSuccess; ++b)
+            e = cudaMemcpy2DAsync(hC + b * d.n * d.n, row, p->stage_c + b * d.stride_c, size_t(d.ldc) * 8, row, size_t(d.n),
+                                  cudaMemcpyDeviceToHost, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "device-to-host copy");
+    return STRASSEN_OK;
+}
+
+void strassen_plan_destroy(strassen_plan *p)
+{
+    if (!p) return;
+    for (TimedLaunch &t : p->pending) {
+        cudaEventDestroy(t.start);
+        cudaEventDestroy(t.stop);
+    }
+    for (cudaEvent_t e : p->free_events) cudaEventDestroy(e);
+    if (p->d_tab) cudaFree(p->d_tab);
+    if (p->own_ws && p->ws) cudaFree(p->ws);
+    if (p->stage_a) cudaFree(p->stage_a);
+    if (p->stage_b) cudaFree(p->stage_b);
+    if (p->stage_c) cudaFree(p->stage_c);
+    delete p;
+}
+
+size_t strassen_plan_workspace_bytes(const strassen_plan *p) { return p ? size_t(p->d.ws_words) * 8 : 0; }
+
+int strassen_plan_set_workspace(strassen_plan *p, void *device_ptr, size_t bytes)
+{
+    g_error.clear();
+    if (!p) return fail(STRASSEN_INVALID_ARG, "plan is NULL");
+    const size_t need = size_t(p->d.ws_words) * 8;
+    if (need == 0) return STRASSEN_OK;
+    if (!device_ptr) return fail(STRASSEN_INVALID_ARG, "workspace pointer is NULL");
+    if (reinterpret_cast<uintptr_t>(device_ptr) & 255) return fail(STRASSEN_MISALIGNED, "workspace must be 256-byte aligned");
+    if (bytes < need) {
+        char buf[128];
+        snprintf(buf, sizeof buf, "workspace of %zu bytes given, %zu needed", bytes, need);
+        return fail(STRASSEN_WORKSPACE_TOO_SMALL, buf);
+    }
+    if (p->own_ws && p->ws) cudaFree(p->ws);
+    p->ws = static_cast<double *>(device_ptr);
+    p->ws_bytes = bytes;
+    p->own_ws = false;
+    return STRASSEN_OK;
+}
+
+const char *strassen_plan_schedule(const strassen_plan *p) { return p ? p->d.schedule.c_str() : ""; }
+int strassen_plan_levels(const strassen_plan *p) { return p ? int(p->d.sizes.size()) - 1 : -1; }
+int64_t strassen_plan_level_size(const strassen_plan *p, int level)
+{
+    if (!p || level < 0 || size_t(level) >= p->d.sizes.size()) return -1;
+    return p->d.sizes[size_t(level)];
+}
+int64_t strassen_plan_base_size(const strassen_plan *p) { return p ? p->d.sizes.back() : -1; }
+int64_t strassen_plan_base_products(const strassen_plan *p)
+{
+    if (!p) return -1;
+    int64_t c = 0;
+    for (const Launch &op : p->d.launches)
+        if (op.kind == OP_GEMM) c += op.count;
+    return c;
+}
+int64_t strassen_plan_launch_count(const strassen_plan *p) { return p ? p->launch_total : -1; }
+int64_t strassen_plan_launches_of(const strassen_plan *p, int kind)
+{
+    if (!p || kind < 0 || kind >= STRASSEN_K_COUNT) return -1;
+    return p->launches[kind];
+}
+
+size_t strassen_schedule_model_bytes(int64_t n, int64_t cutoff, int64_t batch, const char *schedule, int accounting)
+{
+    g_error.clear();
+    if (n < 1 || cutoff < 1 || batch < 1 || !schedule) {
+        fail(STRASSEN_INVALID_ARG, "n, cutoff, batch must be positive and schedule non-NULL");
+        return 0;
+    }
+    const int64_t w = model_workspace_words(level_sizes(n, cutoff), schedule, batch, accounting);
+    if (w < 0) {
+        fail(STRASSEN_BAD_SCHEDULE, "schedule must have one 'B' or 'D' per level and accounting must be 15 or 21");
+        return 0;
+    }
+    return size_t(w) * 8;
+}
+
+int strassen_plan_set_timing(strassen_plan *p, int enabled)
+{
+    if (!p) return fail(STRASSEN_INVALID_ARG, "plan is NULL");
+    p->timing = enabled != 0;
+    return STRASSEN_OK;
+}
+
+int strassen_plan_get_timings(strassen_plan *p, double *ms_out)
+{
+    g_error.clear();
+    if (!p || !ms_out) return fail(STRASSEN_INVALID_ARG, "plan and output must be non-NULL");
+    for (TimedLaunch &t : p->pending) {
+        cudaError_t e = cudaEventSynchronize(t.stop);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, t.start, t.stop);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventElapsedTime");
+        p->acc_ms[t.kind] += double(ms);
+        p->free_events.push_back(t.start);
+        p->free_events.push_back(t.stop);
+    }
+    p->pending.clear();
+    for (int k = 0; k < STRASSEN_K_COUNT; ++k) {
+        ms_out[k] = p->acc_ms[k];
+        p->acc_ms[k] = 0.0;
+    }
+    return STRASSEN_OK;
+}
+
+int strassen_probe_fp64(int kind, int64_t iters, void *stream, double *tflops_out)
+{
+    g_error.clear();
+    if (kind < 0 || kind > 4 || iters < 1 || !tflops_out) return fail(STRASSEN_INVALID_ARG, "kind in 0..4, iters >= 1, output non-NULL");
+    cudaError_t e = probe_fp64(kind, iters, static_cast<cudaStream_t>(stream), tflops_out);
+    if (e != cudaSuccess) return cuda_fail(e, "fp64 probe");
+    return STRASSEN_OK;
+}
+
+const char *strassen_last_error(void) { return g_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,246 @@
+// Batched FP64 base-case products Q = T.S for all live leaves in one launch
+// (Algorithm 2 "localStrassen" at its cutoff; Section 5.4: classical multiply below n0).
+//
+// sm_100a has no FP64 kind in tcgen05.mma, so the tensor-core route for this contraction is
+// the warp-level DMMA (mma.sync m8n8k4, f64 accumulate in registers).  Design:
+//   * persistent CTAs (one per SM, 256 threads = 8 warps as 2 x 4), static round-robin over
+//     the flattened list of 128 x 128 output tiles of all leaves; tiles of one leaf are
+//     adjacent so that CTAs running together share its operand panels through L2;
+//   * operands staged by cp.async into a 4-stage shared-memory ring of 128x16 (A) and
+//     16x128 (B) slabs; the ring runs continuously across tiles, so the loads of the next
+//     tile are in flight while the current one finishes;
+//   * rows padded (+4 doubles) so that the 8-byte fragment loads of a half-warp fall in 16
+//     distinct bank pairs;
+//   * each warp owns 64 x 32 of the tile: 8 x 4 DMMA accumulators of 8 x 8;
+//   * ragged edges (size not a multiple of 128 / 16) are zero-filled by cp.async's src-size
+//     operand and masked in the epilogue; operands that are only 8-byte aligned (views into
+//     matrices with an odd leading dimension) use 8-byte copies.
+#include "kernels.h"
+
+namespace strassen {
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 16, STAGES = 4, THREADS = 256;
+constexpr int AS = BK + 4;            // padded row of the A slab (doubles)
+constexpr int BS = BN + 4;            // padded row of the B slab
+constexpr int A_STAGE = BM * AS;      // 2560 doubles
+constexpr int B_STAGE = BK * BS;      // 2112 doubles
+constexpr int STAGE_WORDS = A_STAGE + B_STAGE;
+constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * sizeof(double);   // 149504
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void dmma_m8n8k4(double &d0, double &d1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
+                 : "+d"(d0), "+d"(d1)
+                 : "d"(a), "d"(b));
+}
+
+struct TileCoord {
+    int node, m0, n0;
+};
+
+__device__ __forceinline__ TileCoord tile_coord(long long t, int tiles_n, int tiles_per_node)
+{
+    TileCoord c;
+    c.node = int(t / tiles_per_node);
+    const int r = int(t - (long long)c.node * tiles_per_node);
+    c.m0 = (r / tiles_n) * BM;
+    c.n0 = (r % tiles_n) * BN;
+    return c;
+}
+
+// Per-thread source state of the tile currently being loaded.
+struct LoadState {
+    const double *a;   // A + (m0 + row0) * lda + kc * 2       (this thread's first chunk, k0 = 0)
+    const double *b;   // B + krow0 * ldb + n0 + nc * 2
+    long long lda, ldb;
+    int a_rows_ok;     // bit i: row m0 + row0 + 32 i < M
+    int b_cols;        // valid columns of this thread's B chunk: 0, 1 or 2
+    bool a16, b16;     // 16-byte copies legal
+};
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n, int tiles_per_node, int ktiles,
+                long long total_tiles)
+{
+    extern __shared__ __align__(16) double smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int wm = warp >> 2, wn = warp & 3;          // 2 x 4 warps
+    const int g = lane >> 2, q = lane & 3;            // DMMA fragment coordinates
+    const uint32_t smem_base = uint32_t(__cvta_generic_to_shared(smem));
+
+    // loader coordinates: A chunk (row, kc) = (tid / 8 + 32 i, tid % 8); B chunk (krow, nc) = (tid / 64 + 4 i, tid % 64)
+    const int a_row0 = tid >> 3, a_kc = tid & 7;
+    const int b_krow0 = tid >> 6, b_nc = tid & 63;
+    const uint32_t a_dst0 = uint32_t((a_row0 * AS + a_kc * 2) * 8);
+    const uint32_t b_dst0 = uint32_t((A_STAGE + b_krow0 * BS + b_nc * 2) * 8);
+
+    long long load_tile = blockIdx.x;
+    int load_k = 0;
+    LoadState ls;
+    const double *safe = reinterpret_cast<const double *>(nodes);
+
+    auto setup_load = [&](long long t) {
+        const TileCoord tc = tile_coord(t, tiles_n, tiles_per_node);
+        const Node nd = nodes[tc.node];
+        const double *A = base_ptr(bases, nd.a.base) + nd.a.off;
+        const double *B = base_ptr(bases, nd.b.base) + nd.b.off;
+        ls.lda = nd.a.ld;
+        ls.ldb = nd.b.ld;
+        ls.a16 = ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && ((nd.a.ld & 1) == 0);
+        ls.b16 = ((reinterpret_cast<uintptr_t>(B) & 15) == 0) && ((nd.b.ld & 1) == 0);
+        ls.a_rows_ok = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (tc.m0 + a_row0 + 32 * i < M) ls.a_rows_ok |= 1 << i;
+        ls.a = A + (long long)(tc.m0 + a_row0) * ls.lda + a_kc * 2;
+        const int col = tc.n0 + b_nc * 2;
+        ls.b_cols = max(0, min(2, M - col));
+        ls.b = B + (long long)b_krow0 * ls.ldb + col;
+    };
+
+    auto issue_load = [&](int stage) {
+        if (load_tile < total_tiles) {
+            if (load_k == 0) setup_load(load_tile);
+            const int k0 = load_k * BK;
+            const uint32_t sbase = smem_base + uint32_t(stage * STAGE_WORDS * 8);
+            // A slab: 128 rows x 16 k.  A copy with src-size 0 reads nothing; it is still given
+            // a valid 16-byte-aligned address (the node table).
+            {
+                const int kvalid = max(0, min(2, M - (k0 + a_kc * 2)));      // K == M (square leaves)
+                const double *src = ls.a + k0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int nv = ((ls.a_rows_ok >> i) & 1) ? kvalid : 0;
+                    const double *s = nv ? src + (long long)(32 * i) * ls.lda : safe;
+                    const uint32_t dst = sbase + a_dst0 + uint32_t(32 * i * AS * 8);
+                    if (ls.a16) {
+                        cp_async16(dst, s, nv * 8);
+                    } else {
+                        cp_async8(dst, s, nv >= 1 ? 8 : 0);
+                        cp_async8(dst + 8, nv >= 2 ? s + 1 : safe, nv >= 2 ? 8 : 0);
+                    }
+                }
+            }
+            // B slab: 16 k x 128 columns
+            {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int nv = (k0 + b_krow0 + 4 * i) < M ? ls.b_cols : 0;
+                    const double *s = nv ? ls.b + (long long)(k0 + 4 * i) * ls.ldb : safe;
+                    const uint32_t dst = sbase + b_dst0 + uint32_t(4 * i * BS * 8);
+                    if (ls.b16) {
+                        cp_async16(dst, s, nv * 8);
+                    } else {
+                        cp_async8(dst, s, nv >= 1 ? 8 : 0);
+                        cp_async8(dst + 8, nv >= 2 ? s + 1 : safe, nv >= 2 ? 8 : 0);
+                    }
+                }
+            }
+            if (++load_k == ktiles) {
+                load_k = 0;
+                load_tile += gridDim.x;
+            }
+        }
+        cp_async_commit();
+    };
+
+    double acc[8][4][2];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) issue_load(s);
+
+    int stage = 0;
+    for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        for (int kt = 0; kt < ktiles; ++kt) {
+            cp_async_wait<STAGES - 2>();
+            __syncthreads();
+            issue_load((stage + STAGES - 1) % STAGES);
+
+            const double *As = smem + stage * STAGE_WORDS + (wm * 64 + g) * AS + q;
+            const double *Bs = smem + stage * STAGE_WORDS + A_STAGE + q * BS + wn * 32 + g;
+#pragma unroll
+            for (int kk = 0; kk < BK / 4; ++kk) {
+                double a[8], b[4];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a[i] = As[i * 8 * AS + kk * 4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) b[j] = Bs[kk * 4 * BS + j * 8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) dmma_m8n8k4(acc[i][j][0], acc[i][j][1], a[i], b[j]);
+            }
+            stage = (stage + 1) % STAGES;
+        }
+        // epilogue: this warp's 64 x 32 block of the tile
+        const TileCoord tc = tile_coord(tile, tiles_n, tiles_per_node);
+        const Node nd = nodes[tc.node];
+        double *C = base_ptr(bases, nd.c.base) + nd.c.off;
+        const long long ldc = nd.c.ld;
+        const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((nd.c.ld & 1) == 0);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = tc.m0 + wm * 64 + i * 8 + g;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int c = tc.n0 + wn * 32 + j * 8 + q * 2;
+                if (r < M && c < M) {
+                    double *o = C + (long long)r * ldc + c;
+                    if (c + 1 < M) {
+                        if (c16) *reinterpret_cast<double2 *>(o) = make_double2(acc[i][j][0], acc[i][j][1]);
+                        else { o[0] = acc[i][j][0]; o[1] = acc[i][j][1]; }
+                    } else {
+                        o[0] = acc[i][j][0];
+                    }
+                }
+                acc[i][j][0] = acc[i][j][1] = 0.0;
+            }
+        }
+    }
+    cp_async_wait<0>();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
+                        int *launched)
+{
+    static bool configured[64] = {false};   // per device: opt in to > 48 KB of dynamic shared memory
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(gemm_f64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(SMEM_BYTES));
+        if (e != cudaSuccess) return e;
+        if (dev < 64) configured[dev] = true;
+    }
+    const int M = int(op.m);
+    const int tiles_m = (M + BM - 1) / BM, tiles_n = (M + BN - 1) / BN;
+    const int tiles_per_node = tiles_m * tiles_n;
+    const int ktiles = (M + BK - 1) / BK;
+    const long long total = (long long)tiles_per_node * op.count;
+    const int grid = int(total < sm_count ? total : sm_count);
+    gemm_f64_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(tab + op.parent_tab, bases, M, tiles_n, tiles_per_node,
+                                                           ktiles, total);
+    ++*launched;
+    return cudaGetLastError();
+}
+
+}  // namespace strassen

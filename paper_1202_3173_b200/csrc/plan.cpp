@@ -1,0 +1,222 @@
+// Host-side planning: level sizes, BFS/DFS schedule against a workspace budget
+// (Limited-Memory rule, Section 3.4), workspace carve-up, node tables and the launch list.
+#include "plan.h"
+
+#include <limits>
+
+namespace strassen {
+
+namespace {
+
+constexpr int64_t kMaxNodes = int64_t(1) << 23;   // table entries (48 B each)
+constexpr int64_t kPadWords = 32;                 // workspace matrices start on 256-byte boundaries
+
+int64_t round_up(int64_t x, int64_t q) { return (x + q - 1) / q * q; }
+
+bool sched_ok(const std::vector<int64_t> &sizes, const std::string &s)
+{
+    if (s.size() + 1 != sizes.size()) return false;
+    for (char c : s)
+        if (c != 'B' && c != 'D') return false;
+    return true;
+}
+
+// The seven operand pairs of a node (Appendix A): which A-side / B-side operand of child j
+// is a plain quadrant (index 0..3 = X11, X12, X21, X22) and which is a computed sum (-1).
+constexpr int kTQuad[7] = {0, 1, -1, -1, -1, -1, 3};   // T0=A11 T1=A12 T6=A22
+constexpr int kSQuad[7] = {0, 2, -1, -1, -1, 3, -1};   // S0=B11 S1=B21 S5=B22
+constexpr int kTSlot[7] = {-1, -1, 0, 1, 2, 3, -1};    // T2..T5 -> slot 0..3
+constexpr int kSSlot[7] = {-1, -1, 0, 1, 2, -1, 3};    // S2,S3,S4,S6 -> slot 0..3
+
+Operand quadrant(const Operand &x, int q, int64_t h)
+{
+    Operand r = x;
+    r.off = x.off + (q & 1 ? h : 0) + (q & 2 ? h * int64_t(x.ld) : 0);
+    return r;
+}
+
+Operand ws_mat(int64_t off, int64_t ldw) { return Operand{off, int32_t(ldw), BASE_WS}; }
+
+bool even(const Operand &x) { return (x.off & 1) == 0 && (x.ld & 1) == 0; }
+
+struct Builder {
+    PlanDesc *p;
+    std::string err;
+
+    int64_t append(const std::vector<Node> &v)
+    {
+        const int64_t at = int64_t(p->nodes.size());
+        if (at + int64_t(v.size()) > kMaxNodes) {
+            err = "recursion tree too large for the node tables (more than 2^23 nodes)";
+            return -1;
+        }
+        p->nodes.insert(p->nodes.end(), v.begin(), v.end());
+        return at;
+    }
+
+    // nodes of `level` are p->nodes[tab .. tab + count)
+    void build(int level, int64_t tab, int64_t count)
+    {
+        if (!err.empty()) return;
+        const int L = int(p->levels.size());
+        if (level == L) {
+            Launch g{};
+            g.kind = OP_GEMM; g.level = level; g.j = -1; g.vec_ok = 1;
+            g.parent_tab = tab; g.child_tab = -1; g.count = count;
+            g.m = p->sizes[level]; g.h = 0;
+            p->launches.push_back(g);
+            return;
+        }
+        const LevelInfo &lv = p->levels[level];
+        const int64_t h = lv.h, mat = lv.mat_words, ldw = lv.ldw, N = count;
+        bool parents_even = (h & 1) == 0;
+        for (int64_t q = 0; q < N; ++q) {
+            const Node &nd = p->nodes[tab + q];
+            parents_even = parents_even && even(nd.a) && even(nd.b) && even(nd.c);
+        }
+        if (lv.mode == 'B') {
+            std::vector<Node> kids(static_cast<size_t>(N) * 7, Node{});
+            const int64_t t_base = lv.ws_off, s_base = lv.ws_off + N * 4 * mat, q_base = lv.ws_off + N * 8 * mat;
+            for (int64_t q = 0; q < N; ++q) {
+                const Node nd = p->nodes[tab + q];
+                for (int j = 0; j < 7; ++j) {
+                    Node &k = kids[size_t(q) * 7 + j];
+                    k.a = kTQuad[j] >= 0 ? quadrant(nd.a, kTQuad[j], h) : ws_mat(t_base + (q * 4 + kTSlot[j]) * mat, ldw);
+                    k.b = kSQuad[j] >= 0 ? quadrant(nd.b, kSQuad[j], h) : ws_mat(s_base + (q * 4 + kSSlot[j]) * mat, ldw);
+                    k.c = ws_mat(q_base + (q * 7 + j) * mat, ldw);
+                }
+            }
+            const int64_t ctab = append(kids);
+            if (ctab < 0) return;
+            Launch f{};
+            f.kind = OP_FORM; f.level = level; f.j = -1; f.vec_ok = parents_even;
+            f.parent_tab = tab; f.child_tab = ctab; f.count = N; f.m = lv.m; f.h = h;
+            p->launches.push_back(f);
+            build(level + 1, ctab, N * 7);
+            Launch r = f;
+            r.kind = OP_RECOMBINE;
+            p->launches.push_back(r);
+        } else {
+            const int64_t t_base = lv.ws_off, s_base = lv.ws_off + N * mat, q_base = lv.ws_off + 2 * N * mat;
+            for (int j = 0; j < 7; ++j) {
+                std::vector<Node> kids(static_cast<size_t>(N), Node{});
+                for (int64_t q = 0; q < N; ++q) {
+                    const Node nd = p->nodes[tab + q];
+                    Node &k = kids[size_t(q)];
+                    k.a = kTQuad[j] >= 0 ? quadrant(nd.a, kTQuad[j], h) : ws_mat(t_base + q * mat, ldw);
+                    k.b = kSQuad[j] >= 0 ? quadrant(nd.b, kSQuad[j], h) : ws_mat(s_base + q * mat, ldw);
+                    k.c = ws_mat(q_base + q * mat, ldw);
+                }
+                const int64_t ctab = append(kids);
+                if (ctab < 0) return;
+                Launch f{};
+                f.kind = OP_FORM_ONE; f.level = level; f.j = j; f.vec_ok = parents_even;
+                f.parent_tab = tab; f.child_tab = ctab; f.count = N; f.m = lv.m; f.h = h;
+                if (kTQuad[j] < 0 || kSQuad[j] < 0) p->launches.push_back(f);   // j = 0, 1 need no sums
+                build(level + 1, ctab, N);
+                Launch a = f;
+                a.kind = OP_ACCUMULATE;
+                p->launches.push_back(a);
+            }
+        }
+        if (lv.peel) {
+            Launch x{};
+            x.kind = OP_PEEL; x.level = level; x.j = -1; x.vec_ok = 0;
+            x.parent_tab = tab; x.child_tab = -1; x.count = N; x.m = lv.m; x.h = h;
+            p->launches.push_back(x);
+        }
+    }
+};
+
+}  // namespace
+
+std::vector<int64_t> level_sizes(int64_t n, int64_t cutoff)
+{
+    std::vector<int64_t> m{n};
+    while (m.back() > cutoff) m.push_back(m.back() / 2);
+    return m;
+}
+
+int64_t actual_workspace_words(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch)
+{
+    if (!sched_ok(sizes, sched)) return -1;
+    int64_t words = 0, live = batch;
+    for (size_t i = 0; i < sched.size(); ++i) {
+        const int64_t h = sizes[i + 1];
+        const int64_t mat = round_up(h * round_up(h, 4), kPadWords);
+        const int64_t per_parent = sched[i] == 'B' ? 15 : 3;
+        if (live > std::numeric_limits<int64_t>::max() / (per_parent * mat) - 1) return std::numeric_limits<int64_t>::max() / 16;
+        words += live * per_parent * mat;
+        if (words < 0 || words > std::numeric_limits<int64_t>::max() / 16) return std::numeric_limits<int64_t>::max() / 16;
+        if (sched[i] == 'B') live *= 7;
+    }
+    return words;
+}
+
+int64_t model_workspace_words(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch,
+                              int accounting)
+{
+    if (!sched_ok(sizes, sched) || (accounting != 15 && accounting != 21)) return -1;
+    long double words = 0;
+    int64_t live = batch;
+    for (size_t i = 0; i < sched.size(); ++i) {
+        const long double h = (long double)sizes[i + 1];
+        words += (long double)live * (sched[i] == 'B' ? accounting : 3) * h * h;
+        if (sched[i] == 'B') live *= 7;
+    }
+    if (words > 1.0e18L) return std::numeric_limits<int64_t>::max() / 16;
+    return int64_t(words);
+}
+
+bool lm_schedule(const std::vector<int64_t> &sizes, int64_t batch, int64_t budget_words, std::string *out)
+{
+    const size_t L = sizes.size() - 1;
+    for (size_t ell = 0; ell <= L; ++ell) {
+        std::string s = std::string(ell, 'D') + std::string(L - ell, 'B');
+        const int64_t w = actual_workspace_words(sizes, s, batch);
+        if (w >= 0 && w <= budget_words) {
+            *out = s;
+            return true;
+        }
+    }
+    return false;
+}
+
+std::string build_plan(PlanDesc *p)
+{
+    if (!sched_ok(p->sizes, p->schedule)) return "schedule does not match the number of levels";
+    const int L = int(p->sizes.size()) - 1;
+    p->levels.clear();
+    p->nodes.clear();
+    p->launches.clear();
+    int64_t live = p->batch, off = 0;
+    for (int i = 0; i < L; ++i) {
+        LevelInfo lv{};
+        lv.m = p->sizes[i];
+        lv.h = p->sizes[i + 1];
+        lv.ldw = round_up(lv.h, 4);
+        lv.mat_words = round_up(lv.h * lv.ldw, kPadWords);
+        lv.parents = live;
+        lv.ws_off = off;
+        lv.mode = p->schedule[i];
+        lv.peel = (lv.m & 1) != 0;
+        off += live * (lv.mode == 'B' ? 15 : 3) * lv.mat_words;
+        if (lv.mode == 'B') live *= 7;
+        if (live > kMaxNodes) return "recursion tree too large for the node tables (more than 2^23 nodes)";
+        p->levels.push_back(lv);
+    }
+    p->ws_words = off;
+
+    std::vector<Node> top(static_cast<size_t>(p->batch), Node{});
+    for (int64_t b = 0; b < p->batch; ++b) {
+        top[size_t(b)].a = Operand{b * p->stride_a, int32_t(p->lda), BASE_A};
+        top[size_t(b)].b = Operand{b * p->stride_b, int32_t(p->ldb), BASE_B};
+        top[size_t(b)].c = Operand{b * p->stride_c, int32_t(p->ldc), BASE_C};
+    }
+    Builder bld{p, {}};
+    const int64_t tab = bld.append(top);
+    if (tab >= 0) bld.build(0, tab, p->batch);
+    return bld.err;
+}
+
+}  // namespace strassen

@@ -1,0 +1,94 @@
+// Internal host-side description of one planned product: level sizes, the resolved
+// BFS/DFS schedule, the workspace carve-up, the node tables and the launch list that
+// strassen_dgemm replays.  Nothing here touches the device.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+namespace strassen {
+
+// Which allocation an operand lives in.  User pointers arrive per call, so the node
+// tables store (base id, element offset, leading dimension) and the kernels resolve
+// addresses from the four base pointers they get as arguments.
+enum Base : int32_t { BASE_A = 0, BASE_B = 1, BASE_C = 2, BASE_WS = 3 };
+
+struct Operand {
+    int64_t off;   // element offset from the base pointer
+    int32_t ld;    // leading dimension in elements
+    int32_t base;  // Base
+};
+
+// One live node of the recursion tree: its two factors and where its product goes.
+struct Node {
+    Operand a, b, c;
+};
+static_assert(sizeof(Node) == 48, "Node is copied to the device as is");
+
+enum OpKind : int32_t {
+    OP_FORM = 0,       // BFS: T2..T5, S2,S3,S4,S6 of `count` parents -> 7*count children
+    OP_GEMM = 1,       // base products of `count` leaves of size m
+    OP_RECOMBINE = 2,  // BFS: 7 Q of each parent -> its four C quadrants
+    OP_FORM_ONE = 3,   // DFS: operands of child j of each parent
+    OP_ACCUMULATE = 4, // DFS: fold Q_j of each parent into its C quadrants
+    OP_PEEL = 5        // odd m: rank-one update, last column, last row
+};
+
+struct Launch {
+    int32_t kind;        // OpKind
+    int32_t level;       // recursion level of the parents (of the leaves for OP_GEMM)
+    int32_t j;           // sub-problem index for OP_FORM_ONE / OP_ACCUMULATE
+    int32_t vec_ok;      // every operand offset and ld involved is even (16-byte accesses
+                         // are legal provided the base pointers are 16-byte aligned)
+    int64_t parent_tab;  // index of the first parent (leaf) node in the table
+    int64_t child_tab;   // index of the first child node (unused for OP_GEMM / OP_PEEL)
+    int64_t count;       // number of parents (leaves)
+    int64_t m;           // size of the parents (leaves)
+    int64_t h;           // size of the children
+};
+
+struct LevelInfo {
+    int64_t m;          // size of a node at this level
+    int64_t h;          // size of its children, floor(m / 2)
+    int64_t ldw;        // leading dimension of the children's workspace matrices
+    int64_t mat_words;  // padded words of one such matrix
+    int64_t parents;    // live nodes at this level (batch * 7^{#B above})
+    int64_t ws_off;     // first word of this level's workspace region
+    char mode;          // 'B' or 'D'
+    bool peel;          // m odd
+};
+
+struct PlanDesc {
+    int64_t n = 0, cutoff = 0, batch = 1;
+    int64_t lda = 0, ldb = 0, ldc = 0;
+    int64_t stride_a = 0, stride_b = 0, stride_c = 0;
+    std::string schedule;           // resolved, one char per level
+    std::vector<int64_t> sizes;     // m_0 .. m_L
+    std::vector<LevelInfo> levels;  // L entries
+    int64_t ws_words = 0;           // total workspace words
+    std::vector<Node> nodes;        // all node tables, concatenated
+    std::vector<Launch> launches;   // replayed in order by strassen_dgemm
+};
+
+// Level sizes m_0 = n, m_{i+1} = floor(m_i / 2) while m_i > cutoff.
+std::vector<int64_t> level_sizes(int64_t n, int64_t cutoff);
+
+// Words of workspace the library itself needs for a schedule (quadrant operands used in
+// place, padded rows); 0 levels -> 0.  Returns -1 if the schedule is malformed.
+int64_t actual_workspace_words(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch);
+
+// Words under the paper's accounting (21 quarter matrices per BFS parent, 3 per DFS parent)
+// or the 15-matrix variant; unpadded.  Returns -1 if the schedule is malformed.
+int64_t model_workspace_words(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch,
+                              int accounting);
+
+// Limited-Memory rule: fewest leading 'D', then 'B' only, that fits budget_words.
+// Returns false if even all-'D' does not fit.
+bool lm_schedule(const std::vector<int64_t> &sizes, int64_t batch, int64_t budget_words, std::string *out);
+
+// Fill levels, workspace layout, node tables and launch list from the scalar fields,
+// sizes and schedule already set in `p`.  Returns an empty string or an error text.
+std::string build_plan(PlanDesc *p);
+
+}  // namespace strassen

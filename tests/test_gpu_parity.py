@@ -1,0 +1,200 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Integer-valued inputs in [-8, 8]: every intermediate is an exact integer, values must be
+equal.  Float inputs: max|C - C_ref| <= 1e-11 * n * max|A| * max|B|, the reference being the
+classical definition computed by the oracle."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1202_3173_b200 import Plan, StrassenError, binding, inputs
+from tests.gpu_util import bound, check_full, check_sampled, run_plan
+
+pytestmark = pytest.mark.gpu
+GB = 1e9
+
+
+def _free_bytes():
+    return torch.cuda.mem_get_info()[0]
+
+
+# ---- base products alone (zero levels), ragged sizes, one and many per launch ----------
+
+@pytest.mark.parametrize("n", [1, 2, 3, 7, 16, 17, 100, 127, 128, 129, 255, 256, 300, 515])
+@pytest.mark.parametrize("dist", ["int8", "uniform"])
+def test_base_product_sizes(n, dist):
+    check_full(n, max(n, 1), "", dist, 100 + n)
+
+
+def test_base_product_batch_spans_many_tiles():
+    check_full(200, 256, "", "int8", 7, batch=40)
+    check_full(384, 512, "", "uniform", 8, batch=9)
+
+
+# ---- tiny recursions: every schedule string -----------------------------------------------
+
+@pytest.mark.parametrize("n,cutoff", [(2, 1), (4, 1), (8, 2), (16, 2), (24, 3), (64, 8)])
+def test_every_schedule_string_small(n, cutoff):
+    L = len(oracle.level_sizes(n, cutoff)) - 1
+    for sched in ("".join(s) for s in itertools.product("BD", repeat=L)):
+        check_full(n, cutoff, sched, "int8", 11 * n + L)
+    check_full(n, cutoff, "B" * L, "uniform", 5 * n)
+    check_full(n, cutoff, "D" * L, "normal", 5 * n + 1)
+
+
+@pytest.mark.parametrize("n,cutoff", [(3, 1), (5, 2), (7, 3), (9, 2), (15, 3), (17, 4), (31, 7), (33, 8), (57, 3),
+                                      (197, 12), (101, 25)])
+def test_peeling_small(n, cutoff):
+    L = len(oracle.level_sizes(n, cutoff)) - 1
+    for sched in {"B" * L, "D" * L, ("BD" * L)[:L], ("DB" * L)[:L]}:
+        check_full(n, cutoff, sched, "int8", 3 * n)
+    check_full(n, cutoff, "B" * L, "uniform", 3 * n + 1)
+
+
+# ---- the small configuration and mid sizes spanning several tiles ---------------------------
+
+def test_config_n512_one_level():
+    check_full(512, 256, "B", "int8", 1002)
+    r = check_full(512, 256, "B", "uniform", 1001)
+    assert r < 1e-3        # calibration: about 1e-5 of the bound at one level
+    check_full(512, 256, "D", "int8", 1002)
+
+
+@pytest.mark.parametrize("n,cutoff,sched", [(1024, 128, "BBB"), (1024, 128, "DBD"), (1024, 128, "BDB"),
+                                            (1024, 256, "DD"), (768, 96, "BBB"), (1000, 125, "DBB"),
+                                            (771, 96, "BBB"), (1543, 192, "BDB"), (2048, 512, "BB")])
+def test_mid_sizes(n, cutoff, sched):
+    check_full(n, cutoff, sched, "int8", n + 1)
+    check_full(n, cutoff, sched, "uniform", n + 2)
+
+
+def test_batch_of_products():
+    check_full(256, 64, "BB", "int8", 21, batch=4)
+    check_full(320, 80, "DB", "uniform", 22, batch=3)
+    check_full(129, 32, "BB", "int8", 23, batch=5)      # odd size inside a batch
+
+
+def test_leading_dimensions_and_strides():
+    n, ld, batch = 96, 101, 2            # odd leading dimension: 8-byte-aligned rows only
+    g = torch.Generator("cuda").manual_seed(5)
+    A = torch.randint(-8, 9, (batch, n + 3, ld), device="cuda", generator=g).double()
+    B = torch.randint(-8, 9, (batch, n + 3, ld), device="cuda", generator=g).double()
+    C = torch.full((batch, n + 3, ld), 777.0, device="cuda", dtype=torch.float64)
+    stride = (n + 3) * ld
+    plan = Plan(n, 12, "BDB", batch=batch, lda=ld, ldb=ld, ldc=ld, stride_a=stride, stride_b=stride, stride_c=stride)
+    ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device="cuda")
+    binding.strassen_plan_set_workspace(plan.handle, ws.data_ptr(), plan.workspace_bytes)
+    binding.strassen_dgemm(plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    plan.close()
+    for b in range(batch):
+        ref = oracle.classical(A[b, :n, :n].cpu().numpy(), B[b, :n, :n].cpu().numpy())
+        assert np.array_equal(C[b, :n, :n].cpu().numpy(), ref)
+    assert bool((C[:, n:, :] == 777.0).all()) and bool((C[:, :, n:] == 777.0).all())   # nothing outside n x n
+
+
+def test_inputs_are_not_written_and_calls_repeat():
+    A, B = inputs.pair(640, "uniform", 31, device="cuda")
+    A0, B0 = A.clone(), B.clone()
+    plan = Plan(640, 80, "BDB")
+    C1 = plan(A, B).clone()
+    C2 = plan(A, B)
+    torch.cuda.synchronize()
+    plan.close()
+    assert torch.equal(A, A0) and torch.equal(B, B0)
+    assert torch.equal(C1, C2)          # same plan, same inputs: same bits
+
+
+def test_schedules_agree_exactly_on_integers():
+    A, B = inputs.pair(512, "int8", 41, device="cuda")
+    outs = [run_plan(512, 64, s, A, B) for s in ("BBB", "DDD", "BDB", "DBD")]
+    for o in outs[1:]:
+        assert torch.equal(outs[0], o)
+
+
+def test_errors_on_device():
+    A, B = inputs.pair(64, "uniform", 1, device="cuda")
+    plan = Plan(64, 16, "BB")
+    with pytest.raises(StrassenError) as e:
+        binding.strassen_dgemm(plan.handle, A.data_ptr(), B.data_ptr(), A.data_ptr(), 0)
+    assert e.value.status == -4
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(StrassenError) as e:
+        binding.strassen_plan_set_workspace(plan.handle, small.data_ptr(), 1024)
+    assert e.value.status == -3
+    plan.close()
+
+
+def test_host_entry_point_copies_in_and_out():
+    n = 384
+    A, B = inputs.pair(n, "int8", 51, device="cpu")
+    A, B = A.pin_memory(), B.pin_memory()
+    C = torch.empty((n, n), dtype=torch.float64).pin_memory()
+    plan = Plan(n, 96, "BB")
+    plan.run_host(A, B, C)
+    torch.cuda.synchronize()
+    plan.close()
+    assert np.array_equal(C.numpy(), oracle.classical(A.numpy(), B.numpy()))
+
+
+def test_timing_split_sums_to_about_the_total():
+    A, B = inputs.pair(2048, "uniform", 61, device="cuda")
+    plan = Plan(2048, 512, "BB")
+    plan(A, B)
+    torch.cuda.synchronize()
+    plan.set_timing(True)
+    plan(A, B)
+    t = plan.timings_ms()
+    plan.close()
+    assert t["gemm"] > 0 and t["form"] > 0 and t["recombine"] > 0 and t["peel"] == 0
+
+
+# ---- full-size configurations: sampled blocks of the definition + exact integer variant ----
+
+def test_config_n4096_bbb_full_size():
+    check_sampled(4096, 512, "BBB", "int8", 2501)
+    r = check_sampled(4096, 512, "BBB", "uniform", 2001)
+    assert r < 1e-2
+
+
+def test_config_batch32_n2048_bb_full_size():
+    if _free_bytes() < 20 * GB:
+        pytest.skip("needs 15 GB")
+    check_sampled(2048, 512, "BB", "int8", 5502, batch=32, members=(0, 13, 31))
+    check_sampled(2048, 512, "BB", "uniform", 5002, batch=32, members=(0, 31))
+
+
+def test_config_n12345_peeling_full_size():
+    if _free_bytes() < 20 * GB:
+        pytest.skip("needs 12 GB")
+    check_sampled(12345, 771, "DBBB", "int8", 5501)
+    check_sampled(12345, 771, "DBBB", "uniform", 5001)
+
+
+def test_config_n16384_dbbbb_full_size():
+    if _free_bytes() < 50 * GB:
+        pytest.skip("needs 31 GB")
+    plan = Plan(16384, 512, "auto", workspace_budget_bytes=int(40 * GB))
+    assert plan.schedule == "DBBBB"
+    plan.close()
+    check_sampled(16384, 512, "DBBBB", "int8", 3501)
+    check_sampled(16384, 512, "DBBBB", "uniform", 3001)
+
+
+def test_config_n47040_full_size():
+    n, cutoff = 47040, 2940
+    abc = 3 * n * n * 8
+    free = _free_bytes()
+    if free < 170 * GB:
+        pytest.skip("needs about 165 GB of device memory")
+    room = int(min(180 * GB, free - 4 * GB) - abc)
+    plan = Plan(n, cutoff, "auto", workspace_budget_bytes=room)
+    sched = plan.schedule
+    plan.close()
+    assert sched in ("DBBB", "DDBB")
+    check_sampled(n, cutoff, sched, "normal", 4001, samples=48)
+    torch.cuda.empty_cache()
+    check_sampled(n, cutoff, sched, "int8", 4501, samples=48)

@@ -1,0 +1,158 @@
+"""Host-side plan logic through the C ABI (no GPU needed): level sizes, schedule strings,
+the Limited-Memory rule, workspace arithmetic against the oracle's memory model and the
+paper's closed forms, launch lists, and error reporting."""
+import itertools
+
+import pytest
+
+import oracle
+from paper_1202_3173_b200 import Plan, StrassenError, binding
+
+GB = 1e9
+
+
+@pytest.mark.parametrize("n,cutoff,L,base", [(512, 256, 1, 256), (4096, 512, 3, 512), (16384, 512, 5, 512),
+                                             (47040, 2940, 4, 2940), (12345, 771, 4, 771), (2048, 512, 2, 512),
+                                             (300, 512, 0, 300), (1, 1, 0, 1), (2, 1, 1, 1)])
+def test_levels_follow_the_cutoff_rule(n, cutoff, L, base):
+    p = Plan(n, cutoff, "B" * L)
+    assert p.levels == L and p.base_size == base
+    assert p.level_sizes == oracle.level_sizes(n, cutoff)
+    assert p.base_products == 7 ** L
+    p.close()
+
+
+def test_schedule_errors():
+    for bad in ("BB", "BBBB", "BXB", "bbb", ""):
+        with pytest.raises(StrassenError) as e:
+            Plan(4096, 512, bad)
+        assert "schedule" in str(e.value)
+    with pytest.raises(StrassenError):
+        Plan(0, 512, "")
+    with pytest.raises(StrassenError):
+        Plan(64, 0, "")
+    with pytest.raises(StrassenError):
+        Plan(64, 8, "BBB", lda=32)
+    with pytest.raises(StrassenError):
+        Plan(64, 8, "BBB", batch=-1)
+
+
+def test_null_arguments_are_reported_not_crashed():
+    l = binding.lib()
+    assert l.strassen_dgemm(None, None, None, None, None) == -1
+    assert b"non-NULL" in l.strassen_last_error()
+    assert l.strassen_plan_create_ex(None) is None
+    l.strassen_plan_destroy(None)
+    assert l.strassen_plan_levels(None) == -1
+    assert l.strassen_plan_workspace_bytes(None) == 0
+
+
+def test_alias_and_alignment_checks_come_before_any_device_work():
+    p = Plan(64, 16, "BB")
+    l = binding.lib()
+    buf = 1 << 20
+    n2 = 64 * 64 * 8
+    assert l.strassen_dgemm(p.handle, buf, buf + n2, buf + n2 // 2, None) == -4      # C overlaps A and B
+    assert l.strassen_dgemm(p.handle, buf, buf + n2, buf + 4, None) == -5          # 4-byte aligned
+    import torch
+    if not torch.cuda.is_available():   # made-up addresses: only where no kernel can run
+        assert l.strassen_dgemm(p.handle, buf, buf, buf + 2 * n2, None) == -6   # A == B is legal; no device
+        assert "cuda" in l.strassen_last_error().decode().lower()
+    p.close()
+
+
+@pytest.mark.parametrize("n,cutoff,batch", [(4096, 512, 1), (16384, 512, 1), (2048, 512, 32), (512, 256, 1)])
+def test_workspace_model_matches_oracle_and_closed_form(n, cutoff, batch):
+    L = len(oracle.level_sizes(n, cutoff)) - 1
+    for sched in ("".join(s) for s in itertools.product("BD", repeat=L)):
+        for acc in (15, 21):
+            assert binding.strassen_schedule_model_bytes(n, cutoff, batch, sched, acc) == \
+                8 * oracle.workspace_words(n, cutoff, sched, batch, acc)
+        p = Plan(n, cutoff, sched, batch=batch)
+        # power-of-two sizes need no padding: the library allocates exactly the 15-matrix figure
+        assert p.workspace_bytes == 8 * oracle.workspace_words(n, cutoff, sched, batch, 15)
+        assert p.schedule == sched
+        p.close()
+    all_b = binding.strassen_schedule_model_bytes(n, cutoff, 1, "B" * L, 21)
+    assert 3 * n * n * 8 + all_b == pytest.approx(8 * oracle.mem_um_closed_form(n, L), rel=1e-13)
+
+
+def test_padded_workspace_for_odd_sizes():
+    n, cutoff, sched = 12345, 771, "DBBB"
+    p = Plan(n, cutoff, sched)
+    lo = 8 * oracle.workspace_words(n, cutoff, sched, 1, 15)
+    assert lo <= p.workspace_bytes <= lo * 1.01
+    assert p.workspace_bytes % 256 == 0
+    p.close()
+
+
+def test_limited_memory_rule():
+    # 16384 under 40 GB: DFS at the top, BFS below
+    p = Plan(16384, 512, "auto", workspace_budget_bytes=int(40 * GB))
+    assert p.schedule == "DBBBB" and p.workspace_bytes <= 40 * GB
+    assert round(p.workspace_bytes / GB, 1) == 24.1
+    p.close()
+    # 47040 with what is left of 180 GB after A, B, C
+    room = int(180 * GB - 3 * 47040 ** 2 * 8)
+    p = Plan(47040, 2940, None, workspace_budget_bytes=room)
+    assert p.schedule == "DBBB" and p.workspace_bytes <= room
+    p.close()
+    # plenty of room: all BFS; tiny room: all DFS; none: error
+    p = Plan(4096, 512, "auto", workspace_budget_bytes=int(10 * GB))
+    assert p.schedule == "BBB"
+    p.close()
+    p = Plan(4096, 512, "auto", workspace_budget_bytes=int(0.14 * GB))
+    assert p.schedule == "DDD"
+    p.close()
+    with pytest.raises(StrassenError):
+        Plan(4096, 512, "auto", workspace_budget_bytes=1000)
+    # an explicit schedule is checked against an explicit budget
+    with pytest.raises(StrassenError):
+        Plan(4096, 512, "BBB", workspace_budget_bytes=int(1 * GB))
+    # same choice as the oracle's statement of the rule, under the library's own accounting
+    for budget_gb in (0.2, 0.5, 1.0, 2.0, 3.0, 5.0):
+        p = Plan(4096, 512, "auto", workspace_budget_bytes=int(budget_gb * GB))
+        assert p.schedule == oracle.lm_schedule(4096, 512, int(budget_gb * GB) // 8, accounting=15)
+        p.close()
+
+
+def test_auto_without_budget_or_device_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    with pytest.raises(StrassenError) as e:
+        Plan(4096, 512, "auto")
+    assert "CUDA" in str(e.value)
+
+
+def test_launch_lists():
+    # all BFS: one form and one recombine per level, one batched product launch
+    p = Plan(4096, 512, "BBB")
+    assert p.launches_by_kind() == {"form": 3, "gemm": 1, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0}
+    assert p.launch_count == 7
+    p.close()
+    # DFS on top: 7 x (form_one [not for j = 0, 1], sub-tree, accumulate)
+    p = Plan(16384, 512, "DBBBB")
+    k = p.launches_by_kind()
+    assert k["form_one"] == 5 and k["accumulate"] == 7 and k["gemm"] == 7 and k["form"] == 28 and k["recombine"] == 28
+    assert p.base_products == 7 ** 5
+    p.close()
+    # all DFS: 7^L single products
+    p = Plan(64, 8, "DDD")
+    assert p.launches_by_kind()["gemm"] == 343 and p.base_products == 343
+    p.close()
+    # peeling adds three fix-up kernels per odd level
+    p = Plan(12345, 771, "BBBB")
+    assert p.launches_by_kind()["peel"] == 6
+    p.close()
+    # zero levels: a single classical product
+    p = Plan(300, 512, "")
+    assert p.launch_count == 1 and p.workspace_bytes == 0
+    p.close()
+
+
+def test_batch_is_extra_live_nodes():
+    p = Plan(2048, 512, "BB", batch=32)
+    assert p.base_products == 32 * 49
+    assert p.launches_by_kind()["gemm"] == 1
+    p.close()
