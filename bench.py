@@ -32,6 +32,10 @@ WORKLOADS = {
     "n47040": (47040, 2940, "auto", 1, "normal", 4001, -1),   # -1: what 180 GB leaves after A, B, C
     "n12345": (12345, 771, "DBBB", 1, "uniform", 5001, 0),
     "b32n2048": (2048, 512, "BB", 32, "uniform", 5002, 0),
+    # the base-product step alone: the 343 leaves of the n=4096 tree as a batch with zero levels
+    "gemm512x343": (512, 512, "", 343, "uniform", 6001, 0),
+    "gemm2940x2": (2940, 2940, "", 2, "uniform", 6002, 0),
+    "gemm771x49": (771, 771, "", 49, "uniform", 6003, 0),
 }
 DEFAULT_WORKLOAD = "n4096"   # the configuration the headline metric is quoted on
 METRIC = "effective FP64 GFLOP/s (2n^3/t)"
@@ -173,6 +177,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
     ap.add_argument("--no-cublas", action="store_true", help="skip the cuBLAS DGEMM comparator")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-probes", action="store_true", help="skip the FP64 rate probes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -230,18 +236,20 @@ def main():
     ms = reduce_max(ms_local, dev)
 
     # ---- end to end: host buffers, copies inside the timed region ----------------------------
-    hA, hB = A.cpu().pin_memory(), B.cpu().pin_memory()
-    hC = torch.empty_like(hA).pin_memory()
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
-        plan.run_host(hA, hB, hC)
-    barrier()
-    ev0.record(stream)
-    for _ in range(e2e_steps):
-        plan.run_host(hA, hB, hC)
-    ev1.record(stream)
-    barrier()
-    e2e_ms = reduce_max(ev0.elapsed_time(ev1) / e2e_steps, dev)
+    e2e_ms = None
+    if not args.no_e2e:
+        hA, hB = A.cpu().pin_memory(), B.cpu().pin_memory()
+        hC = torch.empty_like(hA).pin_memory()
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            plan.run_host(hA, hB, hC)
+        barrier()
+        ev0.record(stream)
+        for _ in range(e2e_steps):
+            plan.run_host(hA, hB, hC)
+        ev1.record(stream)
+        barrier()
+        e2e_ms = reduce_max(ev0.elapsed_time(ev1) / e2e_steps, dev)
 
     if rank != 0:
         plan.close()
@@ -257,6 +265,8 @@ def main():
 
     probes = {}
     for kind, name in enumerate(("dfma", "dmma_m8n8k4", "dmma_m16n8k4", "dmma_m16n8k8", "dmma_m16n8k16")):
+        if args.no_probes:
+            break
         try:
             probes[name] = round(binding.strassen_probe_fp64(kind, 20000, stream.cuda_stream), 2)
         except Exception as exc:   # a probe is context, never fatal
@@ -290,8 +300,8 @@ def main():
     cpu = None
     if not args.no_cpu_baseline:
         import oracle
-        a_h = (hA if batch == 1 else hA[0]).numpy()
-        b_h = (hB if batch == 1 else hB[0]).numpy()
+        a_h = (A if batch == 1 else A[0]).cpu().numpy()
+        b_h = (B if batch == 1 else B[0]).cpu().numpy()
         g, rows, secs = time_oracle_slab(n, a_h, b_h)
         cpu = {"value": g, "unit": UNIT, "cores": oracle.cores(), "kind": "oracle",
                "sample": "classical oracle on the first %d of %d rows of one product (%.1f s); classical flops "
@@ -309,7 +319,8 @@ def main():
                          % (3 * batch * n * n * 8 / 1e6),
                    "parallelism": "replicas only (no collective)" if world > 1 else "single GPU"},
         "clocks": clocks,
-        "e2e": {"value": whole_job_value(n, batch, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": None if e2e_ms is None else
+               {"value": whole_job_value(n, batch, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 2 * batch * n * n * 8, "d2h_bytes_per_step": batch * n * n * 8},
         "gpu_launches": args.steps * plan.launch_count,
         "roofline": {"bound": "alu", "kernel": "gemm_f64_kernel (batched base products)", "achieved": achieved_tflops,
