@@ -2,19 +2,26 @@
 // (Algorithm 2 "localStrassen" at its cutoff; Section 5.4: classical multiply below n0).
 //
 // sm_100a has no FP64 kind in tcgen05.mma, so the tensor-core route for this contraction is
-// the warp-level DMMA (mma.sync m8n8k4, f64 accumulate in registers).  Design:
+// the warp-level DMMA, mma.sync m8n8k4 with FP64 accumulators in registers (the larger f64
+// shapes issue the same number of native 8x8x4 operations and run at the same rate).  Design:
 //   * persistent CTAs (one per SM, 256 threads = 8 warps as 2 x 4), static round-robin over
 //     the flattened list of 128 x 128 output tiles of all leaves; tiles of one leaf are
 //     adjacent so that CTAs running together share its operand panels through L2;
 //   * operands staged by cp.async into a 4-stage shared-memory ring of 128x16 (A) and
 //     16x128 (B) slabs; the ring runs continuously across tiles, so the loads of the next
 //     tile are in flight while the current one finishes;
+//   * one barrier per 16-deep slab, placed before the last quarter of the slab's DMMAs, and
+//     the first fragments of the next slab are read right after it, so that no warp waits
+//     for shared-memory latency with an empty tensor pipe;
 //   * rows padded (+4 doubles) so that the 8-byte fragment loads of a half-warp fall in 16
 //     distinct bank pairs;
 //   * each warp owns 64 x 32 of the tile: 8 x 4 DMMA accumulators of 8 x 8;
-//   * ragged edges (size not a multiple of 128 / 16) are zero-filled by cp.async's src-size
-//     operand and masked in the epilogue; operands that are only 8-byte aligned (views into
-//     matrices with an odd leading dimension) use 8-byte copies.
+//   * interior slabs of 16-byte-aligned operands take a branch-free copy path; ragged edges
+//     (size not a multiple of 128 / 16) are zero-filled by cp.async's src-size operand and
+//     masked in the epilogue; operands that are only 8-byte aligned (views into matrices
+//     with an odd leading dimension) use 8-byte copies.
+#include <cstdlib>
+
 #include "kernels.h"
 
 namespace strassen {
@@ -28,10 +35,15 @@ constexpr int A_STAGE = BM * AS;      // 2560 doubles
 constexpr int B_STAGE = BK * BS;      // 2112 doubles
 constexpr int STAGE_WORDS = A_STAGE + B_STAGE;
 constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * sizeof(double);   // 149504
+static_assert(STAGES == 4, "slot arithmetic below uses & 3");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async16_full(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async8(uint32_t dst, const void *src, int src_bytes)
 {
@@ -40,11 +52,13 @@ __device__ __forceinline__ void cp_async8(uint32_t dst, const void *src, int src
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
-__device__ __forceinline__ void dmma_m8n8k4(double &d0, double &d1, double a, double b)
+// D += A.B, one warp-wide 8x8x4 FP64 tensor-core operation.  g = lane / 4, q = lane % 4:
+// a = A[g][q], b = B[q][g], d0, d1 = D[g][2q], D[g][2q + 1].
+__device__ __forceinline__ void dmma(double &d0, double &d1, double a, double b)
 {
-    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
-                 : "+d"(d0), "+d"(d1)
-                 : "d"(a), "d"(b));
+    asm("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
+        : "+d"(d0), "+d"(d1)
+        : "d"(a), "d"(b));
 }
 
 struct TileCoord {
@@ -61,14 +75,16 @@ __device__ __forceinline__ TileCoord tile_coord(long long t, int tiles_n, int ti
     return c;
 }
 
-// Per-thread source state of the tile currently being loaded.
+// Per-thread source state of the tile currently being loaded; a and b advance slab by slab.
 struct LoadState {
-    const double *a;   // A + (m0 + row0) * lda + kc * 2       (this thread's first chunk, k0 = 0)
-    const double *b;   // B + krow0 * ldb + n0 + nc * 2
-    long long lda, ldb;
-    int a_rows_ok;     // bit i: row m0 + row0 + 32 i < M
-    int b_cols;        // valid columns of this thread's B chunk: 0, 1 or 2
-    bool a16, b16;     // 16-byte copies legal
+    const double *a;        // element (m0 + row0, k0 + 2 kc) of A: this thread's first chunk of the slab
+    const double *b;        // element (k0 + krow0, n0 + 2 nc) of B
+    long long a_step;       // 32 rows of A
+    long long b_step;       // 4 rows of B
+    int a_rows_ok;          // bit i: row m0 + row0 + 32 i < M
+    int b_cols;             // valid columns of this thread's B chunk: 0, 1 or 2
+    bool a16, b16;          // 16-byte copies legal
+    bool interior;          // all rows / columns valid and both operands 16-byte aligned
 };
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -84,48 +100,53 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
     // loader coordinates: A chunk (row, kc) = (tid / 8 + 32 i, tid % 8); B chunk (krow, nc) = (tid / 64 + 4 i, tid % 64)
     const int a_row0 = tid >> 3, a_kc = tid & 7;
     const int b_krow0 = tid >> 6, b_nc = tid & 63;
-    const uint32_t a_dst0 = uint32_t((a_row0 * AS + a_kc * 2) * 8);
-    const uint32_t b_dst0 = uint32_t((A_STAGE + b_krow0 * BS + b_nc * 2) * 8);
+    const uint32_t a_dst0 = smem_base + uint32_t((a_row0 * AS + a_kc * 2) * 8);
+    const uint32_t b_dst0 = smem_base + uint32_t((A_STAGE + b_krow0 * BS + b_nc * 2) * 8);
+    const bool k_ragged = (M % BK) != 0;
 
     long long load_tile = blockIdx.x;
     int load_k = 0;
     LoadState ls;
-    const double *safe = reinterpret_cast<const double *>(nodes);
+    const double *safe = reinterpret_cast<const double *>(nodes);   // valid, 16-byte aligned: for copies of 0 bytes
 
     auto setup_load = [&](long long t) {
         const TileCoord tc = tile_coord(t, tiles_n, tiles_per_node);
         const Node nd = nodes[tc.node];
         const double *A = base_ptr(bases, nd.a.base) + nd.a.off;
         const double *B = base_ptr(bases, nd.b.base) + nd.b.off;
-        ls.lda = nd.a.ld;
-        ls.ldb = nd.b.ld;
+        ls.a_step = 32ll * nd.a.ld;
+        ls.b_step = 4ll * nd.b.ld;
         ls.a16 = ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && ((nd.a.ld & 1) == 0);
         ls.b16 = ((reinterpret_cast<uintptr_t>(B) & 15) == 0) && ((nd.b.ld & 1) == 0);
         ls.a_rows_ok = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             if (tc.m0 + a_row0 + 32 * i < M) ls.a_rows_ok |= 1 << i;
-        ls.a = A + (long long)(tc.m0 + a_row0) * ls.lda + a_kc * 2;
+        ls.a = A + (long long)(tc.m0 + a_row0) * nd.a.ld + a_kc * 2;
         const int col = tc.n0 + b_nc * 2;
         ls.b_cols = max(0, min(2, M - col));
-        ls.b = B + (long long)b_krow0 * ls.ldb + col;
+        ls.b = B + (long long)b_krow0 * nd.b.ld + col;
+        ls.interior = ls.a16 && ls.b16 && tc.m0 + BM <= M && tc.n0 + BN <= M;
     };
 
-    auto issue_load = [&](int stage) {
+    auto issue_load = [&](int slot) {
         if (load_tile < total_tiles) {
             if (load_k == 0) setup_load(load_tile);
-            const int k0 = load_k * BK;
-            const uint32_t sbase = smem_base + uint32_t(stage * STAGE_WORDS * 8);
-            // A slab: 128 rows x 16 k.  A copy with src-size 0 reads nothing; it is still given
-            // a valid 16-byte-aligned address (the node table).
-            {
-                const int kvalid = max(0, min(2, M - (k0 + a_kc * 2)));      // K == M (square leaves)
-                const double *src = ls.a + k0;
+            const uint32_t soff = uint32_t(slot * STAGE_WORDS * 8);
+            if (ls.interior && !(k_ragged && load_k == ktiles - 1)) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) cp_async16_full(a_dst0 + soff + uint32_t(32 * i * AS * 8), ls.a + i * ls.a_step);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) cp_async16_full(b_dst0 + soff + uint32_t(4 * i * BS * 8), ls.b + i * ls.b_step);
+            } else {
+                const int k0 = load_k * BK;
+                // A slab: 128 rows x 16 k (K == M: the leaves are square)
+                const int kvalid = max(0, min(2, M - (k0 + a_kc * 2)));
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int nv = ((ls.a_rows_ok >> i) & 1) ? kvalid : 0;
-                    const double *s = nv ? src + (long long)(32 * i) * ls.lda : safe;
-                    const uint32_t dst = sbase + a_dst0 + uint32_t(32 * i * AS * 8);
+                    const double *s = nv ? ls.a + i * ls.a_step : safe;
+                    const uint32_t dst = a_dst0 + soff + uint32_t(32 * i * AS * 8);
                     if (ls.a16) {
                         cp_async16(dst, s, nv * 8);
                     } else {
@@ -133,14 +154,12 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                         cp_async8(dst + 8, nv >= 2 ? s + 1 : safe, nv >= 2 ? 8 : 0);
                     }
                 }
-            }
-            // B slab: 16 k x 128 columns
-            {
+                // B slab: 16 k x 128 columns
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int nv = (k0 + b_krow0 + 4 * i) < M ? ls.b_cols : 0;
-                    const double *s = nv ? ls.b + (long long)(k0 + 4 * i) * ls.ldb : safe;
-                    const uint32_t dst = sbase + b_dst0 + uint32_t(4 * i * BS * 8);
+                    const double *s = nv ? ls.b + i * ls.b_step : safe;
+                    const uint32_t dst = b_dst0 + soff + uint32_t(4 * i * BS * 8);
                     if (ls.b16) {
                         cp_async16(dst, s, nv * 8);
                     } else {
@@ -149,6 +168,8 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                     }
                 }
             }
+            ls.a += BK;
+            ls.b += 4 * ls.b_step;
             if (++load_k == ktiles) {
                 load_k = 0;
                 load_tile += gridDim.x;
@@ -163,31 +184,49 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
 
+    // fragments of one 4-deep step: A[64 rows of the warp][4 k] and B[4 k][32 columns of the warp]
+    const double *a_frag0 = smem + (wm * 64 + g) * AS + q;
+    const double *b_frag0 = smem + A_STAGE + q * BS + wn * 32 + g;
+    auto load_frags = [&](int slot, int kk, double (&fa)[8], double (&fb)[4]) {
+        const double *As = a_frag0 + slot * STAGE_WORDS + kk * 4;
+        const double *Bs = b_frag0 + slot * STAGE_WORDS + kk * 4 * BS;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) fa[i] = As[i * 8 * AS];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) fb[j] = Bs[j * 8];
+    };
+    auto mma_step = [&](const double (&fa)[8], const double (&fb)[4]) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dmma(acc[i][j][0], acc[i][j][1], fa[i], fb[j]);
+    };
+
 #pragma unroll
     for (int s = 0; s < STAGES - 1; ++s) issue_load(s);
+    cp_async_wait<STAGES - 2>();      // slab 0 has landed
+    __syncthreads();
 
-    int stage = 0;
+    double fa0[8], fb0[4], fa1[8], fb1[4];
+    int slot = 0;
+    load_frags(slot, 0, fa0, fb0);
+
     for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         for (int kt = 0; kt < ktiles; ++kt) {
-            cp_async_wait<STAGES - 2>();
-            __syncthreads();
-            issue_load((stage + STAGES - 1) % STAGES);
-
-            const double *As = smem + stage * STAGE_WORDS + (wm * 64 + g) * AS + q;
-            const double *Bs = smem + stage * STAGE_WORDS + A_STAGE + q * BS + wn * 32 + g;
-#pragma unroll
-            for (int kk = 0; kk < BK / 4; ++kk) {
-                double a[8], b[4];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) a[i] = As[i * 8 * AS + kk * 4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) b[j] = Bs[kk * 4 * BS + j * 8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) dmma_m8n8k4(acc[i][j][0], acc[i][j][1], a[i], b[j]);
-            }
-            stage = (stage + 1) % STAGES;
+            // Invariant: every warp has passed the barrier of the previous slab, i.e. has finished
+            // reading it, so its slot may be refilled; fa0 / fb0 hold step 0 of this slab.
+            load_frags(slot, 1, fa1, fb1);
+            mma_step(fa0, fb0);
+            issue_load((slot + STAGES - 1) & 3);
+            load_frags(slot, 2, fa0, fb0);
+            mma_step(fa1, fb1);
+            load_frags(slot, 3, fa1, fb1);
+            mma_step(fa0, fb0);
+            cp_async_wait<STAGES - 2>();      // this thread's copies of the next slab are complete
+            __syncthreads();                  // ... and everyone's; all reads of this slab are done
+            slot = (slot + 1) & 3;
+            load_frags(slot, 0, fa0, fb0);
+            mma_step(fa1, fb1);
         }
         // epilogue: this warp's 64 x 32 block of the tile
         const TileCoord tc = tile_coord(tile, tiles_n, tiles_per_node);
