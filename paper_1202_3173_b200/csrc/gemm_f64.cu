@@ -28,14 +28,26 @@ namespace strassen {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 16, STAGES = 4, THREADS = 256;
+constexpr int BM = 128, BK = 16;
 constexpr int AS = BK + 4;            // padded row of the A slab (doubles)
-constexpr int BS = BN + 4;            // padded row of the B slab
 constexpr int A_STAGE = BM * AS;      // 2560 doubles
-constexpr int B_STAGE = BK * BS;      // 2112 doubles
-constexpr int STAGE_WORDS = A_STAGE + B_STAGE;
-constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * sizeof(double);   // 149504
-static_assert(STAGES == 4, "slot arithmetic below uses & 3");
+
+// Tile shape variants: BN columns per CTA tile (each warp owns 64 x 32, warps are 2 x BN/32),
+// STAGES slabs in the ring, CTAS resident per SM.
+template <int BN_, int STAGES_, int CTAS_> struct Cfg {
+    static constexpr int BN = BN_, STAGES = STAGES_, CTAS = CTAS_;
+    static constexpr int WARPS_N = BN / 32, THREADS = 2 * WARPS_N * 32;
+    static constexpr int BS = BN + 4;                 // padded row of the B slab
+    static constexpr int B_STAGE = BK * BS;
+    static constexpr int STAGE_WORDS = A_STAGE + B_STAGE;
+    static constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * sizeof(double);
+    static constexpr int A_CHUNKS = BM * (BK / 2) / THREADS;   // 16-byte chunks of the A slab per thread
+    static constexpr int A_ROWS_STEP = THREADS / 8;
+    static constexpr int B_CHUNKS = BK * (BN / 2) / THREADS;   // = 4
+    static_assert(B_CHUNKS == 4, "loader assumes four B chunks per thread");
+};
+using CfgWide = Cfg<128, 4, 1>;     // 149.5 KB of shared memory, one CTA per SM
+using CfgPair = Cfg<64, 3, 2>;      // 87.6 KB, two independent CTAs per SM
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
 {
@@ -65,6 +77,7 @@ struct TileCoord {
     int node, m0, n0;
 };
 
+template <int BN>
 __device__ __forceinline__ TileCoord tile_coord(long long t, int tiles_n, int tiles_per_node)
 {
     TileCoord c;
@@ -79,27 +92,31 @@ __device__ __forceinline__ TileCoord tile_coord(long long t, int tiles_n, int ti
 struct LoadState {
     const double *a;        // element (m0 + row0, k0 + 2 kc) of A: this thread's first chunk of the slab
     const double *b;        // element (k0 + krow0, n0 + 2 nc) of B
-    long long a_step;       // 32 rows of A
+    long long a_step;       // A_ROWS_STEP rows of A
     long long b_step;       // 4 rows of B
-    int a_rows_ok;          // bit i: row m0 + row0 + 32 i < M
+    int a_rows_ok;          // bit i: row m0 + row0 + A_ROWS_STEP i < M
     int b_cols;             // valid columns of this thread's B chunk: 0, 1 or 2
     bool a16, b16;          // 16-byte copies legal
     bool interior;          // all rows / columns valid and both operands 16-byte aligned
 };
 
-__global__ void __launch_bounds__(THREADS, 1)
+template <class C>
+__global__ void __launch_bounds__(C::THREADS, C::CTAS)
 gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n, int tiles_per_node, int ktiles,
                 long long total_tiles)
 {
+    constexpr int BN = C::BN, BS = C::BS, STAGES = C::STAGES, STAGE_WORDS = C::STAGE_WORDS;
+    constexpr int A_CHUNKS = C::A_CHUNKS, A_ROWS_STEP = C::A_ROWS_STEP;
     extern __shared__ __align__(16) double smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int wm = warp >> 2, wn = warp & 3;          // 2 x 4 warps
+    const int wm = warp / C::WARPS_N, wn = warp % C::WARPS_N;   // 2 x WARPS_N warps
     const int g = lane >> 2, q = lane & 3;            // DMMA fragment coordinates
     const uint32_t smem_base = uint32_t(__cvta_generic_to_shared(smem));
 
-    // loader coordinates: A chunk (row, kc) = (tid / 8 + 32 i, tid % 8); B chunk (krow, nc) = (tid / 64 + 4 i, tid % 64)
+    // loader coordinates: A chunk (row, kc) = (tid / 8 + A_ROWS_STEP i, tid % 8);
+    // B chunk (krow, nc) = (tid / (BN / 2) + 4 i, tid % (BN / 2))
     const int a_row0 = tid >> 3, a_kc = tid & 7;
-    const int b_krow0 = tid >> 6, b_nc = tid & 63;
+    const int b_krow0 = tid / (BN / 2), b_nc = tid % (BN / 2);
     const uint32_t a_dst0 = smem_base + uint32_t((a_row0 * AS + a_kc * 2) * 8);
     const uint32_t b_dst0 = smem_base + uint32_t((A_STAGE + b_krow0 * BS + b_nc * 2) * 8);
     const bool k_ragged = (M % BK) != 0;
@@ -109,19 +126,26 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
     LoadState ls;
     const double *safe = reinterpret_cast<const double *>(nodes);   // valid, 16-byte aligned: for copies of 0 bytes
 
-    auto setup_load = [&](long long t) {
-        const TileCoord tc = tile_coord(t, tiles_n, tiles_per_node);
-        const Node nd = nodes[tc.node];
+    // The node of the tile whose loads start next is fetched one slab ahead of its use, so that
+    // the table read never sits between a warp and its next DMMAs.
+    TileCoord next_tc = tile_coord<BN>(load_tile < total_tiles ? load_tile : 0, tiles_n, tiles_per_node);
+    Operand next_a = nodes[next_tc.node].a, next_b = nodes[next_tc.node].b;
+
+    auto setup_load = [&]() {
+        const TileCoord tc = next_tc;
+        Node nd;
+        nd.a = next_a;
+        nd.b = next_b;
         const double *A = base_ptr(bases, nd.a.base) + nd.a.off;
         const double *B = base_ptr(bases, nd.b.base) + nd.b.off;
-        ls.a_step = 32ll * nd.a.ld;
+        ls.a_step = (long long)A_ROWS_STEP * nd.a.ld;
         ls.b_step = 4ll * nd.b.ld;
         ls.a16 = ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && ((nd.a.ld & 1) == 0);
         ls.b16 = ((reinterpret_cast<uintptr_t>(B) & 15) == 0) && ((nd.b.ld & 1) == 0);
         ls.a_rows_ok = 0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (tc.m0 + a_row0 + 32 * i < M) ls.a_rows_ok |= 1 << i;
+        for (int i = 0; i < A_CHUNKS; ++i)
+            if (tc.m0 + a_row0 + A_ROWS_STEP * i < M) ls.a_rows_ok |= 1 << i;
         ls.a = A + (long long)(tc.m0 + a_row0) * nd.a.ld + a_kc * 2;
         const int col = tc.n0 + b_nc * 2;
         ls.b_cols = max(0, min(2, M - col));
@@ -131,11 +155,12 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
 
     auto issue_load = [&](int slot) {
         if (load_tile < total_tiles) {
-            if (load_k == 0) setup_load(load_tile);
+            if (load_k == 0) setup_load();
             const uint32_t soff = uint32_t(slot * STAGE_WORDS * 8);
             if (ls.interior && !(k_ragged && load_k == ktiles - 1)) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) cp_async16_full(a_dst0 + soff + uint32_t(32 * i * AS * 8), ls.a + i * ls.a_step);
+                for (int i = 0; i < A_CHUNKS; ++i)
+                    cp_async16_full(a_dst0 + soff + uint32_t(A_ROWS_STEP * i * AS * 8), ls.a + i * ls.a_step);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) cp_async16_full(b_dst0 + soff + uint32_t(4 * i * BS * 8), ls.b + i * ls.b_step);
             } else {
@@ -143,10 +168,10 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                 // A slab: 128 rows x 16 k (K == M: the leaves are square)
                 const int kvalid = max(0, min(2, M - (k0 + a_kc * 2)));
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < A_CHUNKS; ++i) {
                     const int nv = ((ls.a_rows_ok >> i) & 1) ? kvalid : 0;
                     const double *s = nv ? ls.a + i * ls.a_step : safe;
-                    const uint32_t dst = a_dst0 + soff + uint32_t(32 * i * AS * 8);
+                    const uint32_t dst = a_dst0 + soff + uint32_t(A_ROWS_STEP * i * AS * 8);
                     if (ls.a16) {
                         cp_async16(dst, s, nv * 8);
                     } else {
@@ -173,6 +198,11 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
             if (++load_k == ktiles) {
                 load_k = 0;
                 load_tile += gridDim.x;
+                if (load_tile < total_tiles) {
+                    next_tc = tile_coord<BN>(load_tile, tiles_n, tiles_per_node);
+                    next_a = nodes[next_tc.node].a;
+                    next_b = nodes[next_tc.node].b;
+                }
             }
         }
         cp_async_commit();
@@ -212,28 +242,28 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
     load_frags(slot, 0, fa0, fb0);
 
     for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const TileCoord tc = tile_coord<BN>(tile, tiles_n, tiles_per_node);
+        const Operand c_op = nodes[tc.node].c;        // consumed after the k loop
         for (int kt = 0; kt < ktiles; ++kt) {
             // Invariant: every warp has passed the barrier of the previous slab, i.e. has finished
             // reading it, so its slot may be refilled; fa0 / fb0 hold step 0 of this slab.
             load_frags(slot, 1, fa1, fb1);
             mma_step(fa0, fb0);
-            issue_load((slot + STAGES - 1) & 3);
+            issue_load((slot + STAGES - 1) % STAGES);
             load_frags(slot, 2, fa0, fb0);
             mma_step(fa1, fb1);
             load_frags(slot, 3, fa1, fb1);
             mma_step(fa0, fb0);
             cp_async_wait<STAGES - 2>();      // this thread's copies of the next slab are complete
             __syncthreads();                  // ... and everyone's; all reads of this slab are done
-            slot = (slot + 1) & 3;
+            slot = slot + 1 == STAGES ? 0 : slot + 1;
             load_frags(slot, 0, fa0, fb0);
             mma_step(fa1, fb1);
         }
         // epilogue: this warp's 64 x 32 block of the tile
-        const TileCoord tc = tile_coord(tile, tiles_n, tiles_per_node);
-        const Node nd = nodes[tc.node];
-        double *C = base_ptr(bases, nd.c.base) + nd.c.off;
-        const long long ldc = nd.c.ld;
-        const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((nd.c.ld & 1) == 0);
+        double *C = base_ptr(bases, c_op.base) + c_op.off;
+        const long long ldc = c_op.ld;
+        const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((c_op.ld & 1) == 0);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int r = tc.m0 + wm * 64 + i * 8 + g;
@@ -258,28 +288,42 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
 
 }  // namespace
 
-cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
-                        int *launched)
+namespace {
+
+template <class C>
+cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, long long count, int sm_count, cudaStream_t stream)
 {
     static bool configured[64] = {false};   // per device: opt in to > 48 KB of dynamic shared memory
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(gemm_f64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(SMEM_BYTES));
+        e = cudaFuncSetAttribute(gemm_f64_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::SMEM_BYTES));
         if (e != cudaSuccess) return e;
         if (dev < 64) configured[dev] = true;
     }
-    const int M = int(op.m);
-    const int tiles_m = (M + BM - 1) / BM, tiles_n = (M + BN - 1) / BN;
+    const int tiles_m = (M + BM - 1) / BM, tiles_n = (M + C::BN - 1) / C::BN;
     const int tiles_per_node = tiles_m * tiles_n;
     const int ktiles = (M + BK - 1) / BK;
-    const long long total = (long long)tiles_per_node * op.count;
-    const int grid = int(total < sm_count ? total : sm_count);
-    gemm_f64_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(tab + op.parent_tab, bases, M, tiles_n, tiles_per_node,
-                                                           ktiles, total);
-    ++*launched;
+    const long long total = (long long)tiles_per_node * count;
+    const long long slots = (long long)sm_count * C::CTAS;
+    const int grid = int(total < slots ? total : slots);
+    gemm_f64_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(nodes, bases, M, tiles_n, tiles_per_node, ktiles, total);
     return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
+                        int *launched)
+{
+    static const int variant = [] {
+        const char *v = getenv("STRASSEN_GEMM_VARIANT");
+        return v ? atoi(v) : 0;
+    }();
+    ++*launched;
+    if (variant == 1) return launch_cfg<CfgPair>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
+    return launch_cfg<CfgWide>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
 }
 
 }  // namespace strassen

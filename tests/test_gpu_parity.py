@@ -18,6 +18,7 @@ GB = 1e9
 
 
 def _free_bytes():
+    torch.cuda.empty_cache()        # memory cached by earlier tests counts as free
     return torch.cuda.mem_get_info()[0]
 
 
