@@ -178,6 +178,47 @@ int strassen_plan_get_timings(strassen_plan *plan, double *ms_out /* [STRASSEN_K
  */
 int strassen_probe_fp64(int kind, int64_t iters, void *stream, double *tflops_out);
 
+/*
+ * strassen_dgemm_static -- C = A.B for one n x n product, 2 <= n <= STRASSEN_STATIC_MAX_N, WITHOUT
+ * allocating anything.  (The paper has no counterpart: this entry point exists for deployment
+ * reasons only.)
+ *
+ * Who it is for: callers that are not allowed to call cudaMalloc / cudaFree when they need a
+ * product -- code running under an allocator that has already claimed the whole device and
+ * hands out no raw memory, latency-critical loops that cannot afford the device-wide
+ * synchronisation an allocation or a free implies, and plug-ins invoked from another library's
+ * callback whose contract forbids allocating.  strassen_dgemm cannot serve them: its plan keeps
+ * node tables and (unless given one) a workspace in memory it obtains from cudaMalloc.
+ *
+ * What it computes: exactly one Strassen-Winograd level (a BFS step, with peeling when n is
+ * odd) over base products of size floor(n / 2), using the same kernels as strassen_dgemm with
+ * cutoff floor(n / 2); the results are identical to that call's.
+ *
+ * Where the temporaries live: the eight operand sums, the seven products and a small node
+ * table are kept in a static device array compiled into the library (about 7.9 MB, sized for
+ * n = STRASSEN_STATIC_MAX_N).  Every GPU that loads the library holds that array until the
+ * process exits.  A larger n is rejected with STRASSEN_WORKSPACE_TOO_SMALL and a message that
+ * names the limit; nothing is launched in that case.
+ *
+ * Arguments: A, B, C device pointers, row-major with contiguous rows (ld = n), 8-byte aligned,
+ * C not overlapping A or B; A and B are only read, C is fully overwritten; stream is a
+ * cudaStream_t passed as void* (NULL = legacy default stream).  Asynchronous like
+ * strassen_dgemm.  Errors are reported the same way (status + strassen_last_error()).
+ *
+ * Rules that follow from the shared array:
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and the SM count; make that first call
+ *     before starting any stream capture on that device.  Later calls do no set-up.
+ *   - All calls on a device use the same array, and it keeps whatever the previous call left
+ *     in it.  No part of it needs to start at zero: every temporary is written in full before
+ *     it is read.  Two calls whose kernels can overlap on the GPU (different streams without
+ *     an ordering between them, or different host threads doing that) would overwrite each
+ *     other's temporaries: order them on one stream or with events.
+ *   - The function calls no cudaMalloc, cudaFree, or any routine that allocates device memory.
+ */
+#define STRASSEN_STATIC_MAX_N 512
+int strassen_dgemm_static(int64_t n, const double *A, const double *B, double *C, void *stream);
+
 /* Text describing the last failure on the calling thread ("" if none).  Thread-local. */
 const char *strassen_last_error(void);
 

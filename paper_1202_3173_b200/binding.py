@@ -49,8 +49,10 @@ SYMBOLS = [
     ("strassen_plan_set_timing", _int, [_vp, _int]),
     ("strassen_plan_get_timings", _int, [_vp, _dp]),
     ("strassen_probe_fp64", _int, [_int, _i64, _vp, _dp]),
+    ("strassen_dgemm_static", _int, [_i64, _vp, _vp, _vp, _vp]),
     ("strassen_last_error", _cp, []),
 ]
+STRASSEN_STATIC_MAX_N = 512
 
 _lib = None
 
@@ -171,6 +173,12 @@ def strassen_plan_get_timings(plan: int):
     out = (ctypes.c_double * K_COUNT)()
     _check(lib().strassen_plan_get_timings(plan, out))
     return dict(zip(KERNEL_KINDS, list(out)))
+
+
+def strassen_dgemm_static(n: int, A: int, B: int, C: int, stream: int = 0) -> None:
+    """One Strassen-Winograd level with all temporaries in the library's static device array:
+    for callers that must not allocate device memory.  A, B, C: device addresses, rows of n."""
+    _check(lib().strassen_dgemm_static(n, A, B, C, stream))
 
 
 def strassen_probe_fp64(kind: int, iters: int, stream: int = 0) -> float:

@@ -212,6 +212,10 @@ strassen_plan *create(const strassen_options &o)
 
 }  // namespace
 
+namespace strassen {
+void set_last_error(const char *msg) { g_error = msg ? msg : ""; }
+}  // namespace strassen
+
 extern "C" {
 
 strassen_plan *strassen_plan_create(int64_t n, int64_t cutoff, const char *schedule)

@@ -36,4 +36,7 @@ int launches_of(const Launch &op);
 
 cudaError_t probe_fp64(int kind, long long iters, cudaStream_t stream, double *tflops_out);
 
+// Sets the calling thread's error text (what strassen_last_error() returns).
+void set_last_error(const char *msg);
+
 }  // namespace strassen
