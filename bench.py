@@ -41,6 +41,10 @@ DEFAULT_WORKLOAD = "n4096"   # the configuration the headline metric is quoted o
 METRIC = "effective FP64 GFLOP/s (2n^3/t)"
 UNIT = "GFLOP/s"
 
+# DRAM bytes (read + write) of the dominant kernel's launch from one ncu capture, per workload
+# (profiles/gemm_f64_kernel_343x512.md); None where no capture of that exact launch exists.
+GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.127e9, "gemm512x343": 2.127e9}
+
 # FP64 arithmetic peak from unit counts and clocks: 148 SMs x 64 FP64 FMA lanes x 2 flop x 1.965 GHz
 FP64_PEAK_NOMINAL_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
 
@@ -327,7 +331,8 @@ def main():
                      "peak": FP64_PEAK_NOMINAL_TFLOPS, "unit": "TFLOP/s", "frac": achieved_tflops / FP64_PEAK_NOMINAL_TFLOPS,
                      "peak_source": "148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz (unit counts and max clock)",
                      "fp64_probe_tflops": probes, "frac_of_probe": achieved_tflops / fp64_measured,
-                     "ms_per_launch": gemm_ms, "flops_per_launch": f_base / gemm_launches, "traffic": None},
+                     "ms_per_launch": gemm_ms, "flops_per_launch": f_base / gemm_launches,
+                     "traffic": GEMM_DRAM_TRAFFIC_BYTES.get(args.workload)},
         "path_roofline": {"t_roof_ms": t_roof_ms, "frac": t_roof_ms / ms_local, "base_flops": f_base, "add_bytes": b_alg,
                           "hbm_gbs": hbm_gbs, "hbm_source": hbm_src,
                           "kernel_ms_per_step": {k: v / args.steps for k, v in kinds.items()}},

@@ -28,26 +28,28 @@ namespace strassen {
 
 namespace {
 
-constexpr int BM = 128, BK = 16;
-constexpr int AS = BK + 4;            // padded row of the A slab (doubles)
-constexpr int A_STAGE = BM * AS;      // 2560 doubles
+constexpr int BM = 128;
 
 // Tile shape variants: BN columns per CTA tile (each warp owns 64 x 32, warps are 2 x BN/32),
-// STAGES slabs in the ring, CTAS resident per SM.
-template <int BN_, int STAGES_, int CTAS_> struct Cfg {
-    static constexpr int BN = BN_, STAGES = STAGES_, CTAS = CTAS_;
+// BK-deep slabs, STAGES slabs in the ring, CTAS resident per SM.
+template <int BN_, int BK_, int STAGES_, int CTAS_> struct Cfg {
+    static constexpr int BN = BN_, BK = BK_, STAGES = STAGES_, CTAS = CTAS_;
     static constexpr int WARPS_N = BN / 32, THREADS = 2 * WARPS_N * 32;
+    static constexpr int AS = BK + 4;                 // padded row of the A slab (doubles)
     static constexpr int BS = BN + 4;                 // padded row of the B slab
-    static constexpr int B_STAGE = BK * BS;
+    static constexpr int A_STAGE = BM * AS, B_STAGE = BK * BS;
     static constexpr int STAGE_WORDS = A_STAGE + B_STAGE;
     static constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * sizeof(double);
-    static constexpr int A_CHUNKS = BM * (BK / 2) / THREADS;   // 16-byte chunks of the A slab per thread
-    static constexpr int A_ROWS_STEP = THREADS / 8;
-    static constexpr int B_CHUNKS = BK * (BN / 2) / THREADS;   // = 4
-    static_assert(B_CHUNKS == 4, "loader assumes four B chunks per thread");
+    static constexpr int A_KCHUNKS = BK / 2;                    // 16-byte chunks per A row
+    static constexpr int A_ROWS_STEP = THREADS / A_KCHUNKS;     // rows covered by one pass of all threads
+    static constexpr int A_CHUNKS = BM / A_ROWS_STEP;           // passes (chunks per thread) for the A slab
+    static constexpr int B_KROWS_STEP = THREADS / (BN / 2);     // B rows covered by one pass
+    static constexpr int B_CHUNKS = BK / B_KROWS_STEP;          // passes for the B slab
+    static_assert(BK % 8 == 0 && AS % 16 == 4 && BS % 16 == 4, "fragment loads rely on stride = 4 mod 16");
 };
-using CfgWide = Cfg<128, 4, 1>;     // 149.5 KB of shared memory, one CTA per SM
-using CfgPair = Cfg<64, 3, 2>;      // 87.6 KB, two independent CTAs per SM
+using CfgWide = Cfg<128, 16, 4, 1>;     // 149.5 KB of shared memory, one CTA per SM
+using CfgPair = Cfg<64, 16, 3, 2>;      // 87.6 KB, two independent CTAs per SM
+using CfgDeep = Cfg<128, 32, 3, 1>;     // 212 KB: half as many barriers per tile
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
 {
@@ -93,7 +95,7 @@ struct LoadState {
     const double *a;        // element (m0 + row0, k0 + 2 kc) of A: this thread's first chunk of the slab
     const double *b;        // element (k0 + krow0, n0 + 2 nc) of B
     long long a_step;       // A_ROWS_STEP rows of A
-    long long b_step;       // 4 rows of B
+    long long b_step;       // B_KROWS_STEP rows of B
     int a_rows_ok;          // bit i: row m0 + row0 + A_ROWS_STEP i < M
     int b_cols;             // valid columns of this thread's B chunk: 0, 1 or 2
     bool a16, b16;          // 16-byte copies legal
@@ -105,17 +107,18 @@ __global__ void __launch_bounds__(C::THREADS, C::CTAS)
 gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n, int tiles_per_node, int ktiles,
                 long long total_tiles)
 {
-    constexpr int BN = C::BN, BS = C::BS, STAGES = C::STAGES, STAGE_WORDS = C::STAGE_WORDS;
-    constexpr int A_CHUNKS = C::A_CHUNKS, A_ROWS_STEP = C::A_ROWS_STEP;
+    constexpr int BN = C::BN, BK = C::BK, AS = C::AS, BS = C::BS, STAGES = C::STAGES, STAGE_WORDS = C::STAGE_WORDS;
+    constexpr int A_STAGE = C::A_STAGE, A_CHUNKS = C::A_CHUNKS, A_ROWS_STEP = C::A_ROWS_STEP, A_KCHUNKS = C::A_KCHUNKS;
+    constexpr int B_CHUNKS = C::B_CHUNKS, B_KROWS_STEP = C::B_KROWS_STEP;
     extern __shared__ __align__(16) double smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int wm = warp / C::WARPS_N, wn = warp % C::WARPS_N;   // 2 x WARPS_N warps
     const int g = lane >> 2, q = lane & 3;            // DMMA fragment coordinates
     const uint32_t smem_base = uint32_t(__cvta_generic_to_shared(smem));
 
-    // loader coordinates: A chunk (row, kc) = (tid / 8 + A_ROWS_STEP i, tid % 8);
-    // B chunk (krow, nc) = (tid / (BN / 2) + 4 i, tid % (BN / 2))
-    const int a_row0 = tid >> 3, a_kc = tid & 7;
+    // loader coordinates: A chunk (row, kc) = (tid / A_KCHUNKS + A_ROWS_STEP i, tid % A_KCHUNKS);
+    // B chunk (krow, nc) = (tid / (BN / 2) + B_KROWS_STEP i, tid % (BN / 2))
+    const int a_row0 = tid / A_KCHUNKS, a_kc = tid % A_KCHUNKS;
     const int b_krow0 = tid / (BN / 2), b_nc = tid % (BN / 2);
     const uint32_t a_dst0 = smem_base + uint32_t((a_row0 * AS + a_kc * 2) * 8);
     const uint32_t b_dst0 = smem_base + uint32_t((A_STAGE + b_krow0 * BS + b_nc * 2) * 8);
@@ -139,7 +142,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
         const double *A = base_ptr(bases, nd.a.base) + nd.a.off;
         const double *B = base_ptr(bases, nd.b.base) + nd.b.off;
         ls.a_step = (long long)A_ROWS_STEP * nd.a.ld;
-        ls.b_step = 4ll * nd.b.ld;
+        ls.b_step = (long long)B_KROWS_STEP * nd.b.ld;
         ls.a16 = ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && ((nd.a.ld & 1) == 0);
         ls.b16 = ((reinterpret_cast<uintptr_t>(B) & 15) == 0) && ((nd.b.ld & 1) == 0);
         ls.a_rows_ok = 0;
@@ -162,7 +165,8 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                 for (int i = 0; i < A_CHUNKS; ++i)
                     cp_async16_full(a_dst0 + soff + uint32_t(A_ROWS_STEP * i * AS * 8), ls.a + i * ls.a_step);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) cp_async16_full(b_dst0 + soff + uint32_t(4 * i * BS * 8), ls.b + i * ls.b_step);
+                for (int i = 0; i < B_CHUNKS; ++i)
+                    cp_async16_full(b_dst0 + soff + uint32_t(B_KROWS_STEP * i * BS * 8), ls.b + i * ls.b_step);
             } else {
                 const int k0 = load_k * BK;
                 // A slab: 128 rows x 16 k (K == M: the leaves are square)
@@ -181,10 +185,10 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                 }
                 // B slab: 16 k x 128 columns
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int nv = (k0 + b_krow0 + 4 * i) < M ? ls.b_cols : 0;
+                for (int i = 0; i < B_CHUNKS; ++i) {
+                    const int nv = (k0 + b_krow0 + B_KROWS_STEP * i) < M ? ls.b_cols : 0;
                     const double *s = nv ? ls.b + i * ls.b_step : safe;
-                    const uint32_t dst = b_dst0 + soff + uint32_t(4 * i * BS * 8);
+                    const uint32_t dst = b_dst0 + soff + uint32_t(B_KROWS_STEP * i * BS * 8);
                     if (ls.b16) {
                         cp_async16(dst, s, nv * 8);
                     } else {
@@ -194,7 +198,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                 }
             }
             ls.a += BK;
-            ls.b += 4 * ls.b_step;
+            ls.b += B_CHUNKS * ls.b_step;
             if (++load_k == ktiles) {
                 load_k = 0;
                 load_tile += gridDim.x;
@@ -247,39 +251,57 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
         for (int kt = 0; kt < ktiles; ++kt) {
             // Invariant: every warp has passed the barrier of the previous slab, i.e. has finished
             // reading it, so its slot may be refilled; fa0 / fb0 hold step 0 of this slab.
-            load_frags(slot, 1, fa1, fb1);
-            mma_step(fa0, fb0);
-            issue_load((slot + STAGES - 1) % STAGES);
-            load_frags(slot, 2, fa0, fb0);
-            mma_step(fa1, fb1);
-            load_frags(slot, 3, fa1, fb1);
-            mma_step(fa0, fb0);
-            cp_async_wait<STAGES - 2>();      // this thread's copies of the next slab are complete
-            __syncthreads();                  // ... and everyone's; all reads of this slab are done
-            slot = slot + 1 == STAGES ? 0 : slot + 1;
-            load_frags(slot, 0, fa0, fb0);
-            mma_step(fa1, fb1);
+#pragma unroll
+            for (int kk = 0; kk < BK / 4; kk += 2) {
+                load_frags(slot, kk + 1, fa1, fb1);
+                mma_step(fa0, fb0);
+                if (kk == 0) issue_load((slot + STAGES - 1) % STAGES);
+                if (kk + 2 < BK / 4) {
+                    load_frags(slot, kk + 2, fa0, fb0);
+                } else {
+                    cp_async_wait<STAGES - 2>();      // this thread's copies of the next slab are complete
+                    __syncthreads();                  // ... and everyone's; all reads of this slab are done
+                    slot = slot + 1 == STAGES ? 0 : slot + 1;
+                    load_frags(slot, 0, fa0, fb0);
+                }
+                mma_step(fa1, fb1);
+            }
         }
         // epilogue: this warp's 64 x 32 block of the tile
         double *C = base_ptr(bases, c_op.base) + c_op.off;
         const long long ldc = c_op.ld;
         const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((c_op.ld & 1) == 0);
+        const int r0 = tc.m0 + wm * 64 + g, c0 = tc.n0 + wn * 32 + q * 2;
+        double *o = C + (long long)r0 * ldc + c0;
+        if (c16 && tc.m0 + BM <= M && tc.n0 + BN <= M) {
+            // interior tile: 16-byte stores at fixed offsets from one running row pointer
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = tc.m0 + wm * 64 + i * 8 + g;
+            for (int i = 0; i < 8; ++i) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int c = tc.n0 + wn * 32 + j * 8 + q * 2;
-                if (r < M && c < M) {
-                    double *o = C + (long long)r * ldc + c;
-                    if (c + 1 < M) {
-                        if (c16) *reinterpret_cast<double2 *>(o) = make_double2(acc[i][j][0], acc[i][j][1]);
-                        else { o[0] = acc[i][j][0]; o[1] = acc[i][j][1]; }
-                    } else {
-                        o[0] = acc[i][j][0];
-                    }
+                for (int j = 0; j < 4; ++j) {
+                    *reinterpret_cast<double2 *>(o + j * 8) = make_double2(acc[i][j][0], acc[i][j][1]);
+                    acc[i][j][0] = acc[i][j][1] = 0.0;
                 }
-                acc[i][j][0] = acc[i][j][1] = 0.0;
+                o += 8 * ldc;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = r0 + i * 8;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int c = c0 + j * 8;
+                    if (r < M && c < M) {
+                        double *e = o + (long long)(i * 8) * ldc + j * 8;
+                        if (c + 1 < M) {
+                            if (c16) *reinterpret_cast<double2 *>(e) = make_double2(acc[i][j][0], acc[i][j][1]);
+                            else { e[0] = acc[i][j][0]; e[1] = acc[i][j][1]; }
+                        } else {
+                            e[0] = acc[i][j][0];
+                        }
+                    }
+                    acc[i][j][0] = acc[i][j][1] = 0.0;
+                }
             }
         }
     }
@@ -304,7 +326,7 @@ cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, long long c
     }
     const int tiles_m = (M + BM - 1) / BM, tiles_n = (M + C::BN - 1) / C::BN;
     const int tiles_per_node = tiles_m * tiles_n;
-    const int ktiles = (M + BK - 1) / BK;
+    const int ktiles = (M + C::BK - 1) / C::BK;
     const long long total = (long long)tiles_per_node * count;
     const long long slots = (long long)sm_count * C::CTAS;
     const int grid = int(total < slots ? total : slots);
@@ -323,6 +345,7 @@ cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, i
     }();
     ++*launched;
     if (variant == 1) return launch_cfg<CfgPair>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
+    if (variant == 2) return launch_cfg<CfgDeep>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
     return launch_cfg<CfgWide>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
 }
 
