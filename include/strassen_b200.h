@@ -75,7 +75,13 @@ typedef struct strassen_options {
     int64_t stride_a, stride_b, stride_c; /* element distance between batch members; 0 means ld * n */
     size_t workspace_budget_bytes;  /* for "auto": largest workspace allowed; 0 = free device memory
                                        of the current device minus a 1 GiB margin                  */
+    int64_t flags;          /* STRASSEN_FLAG_* bits; 0 = defaults                                  */
 } strassen_options;
+
+/* By default two consecutive BFS levels are formed and recombined in one pass each (the children's
+ * operands are not read back and their products never written: fewer HBM bytes, same arithmetic in
+ * the same order, bit-identical results).  This flag keeps one pass per level. */
+#define STRASSEN_FLAG_SINGLE_LEVEL_PASSES 1
 
 /*
  * strassen_plan_create -- plan C = A.B for n x n matrices [Algorithm 1 "Require A, B n x n"].

@@ -21,10 +21,10 @@ class Plan:
     """
 
     def __init__(self, n, cutoff, schedule=None, batch=1, workspace_budget_bytes=0, lda=0, ldb=0, ldc=0,
-                 stride_a=0, stride_b=0, stride_c=0):
+                 stride_a=0, stride_b=0, stride_c=0, flags=0):
         self.n, self.cutoff, self.batch = int(n), int(cutoff), int(batch)
         self._h = binding.strassen_plan_create_ex(n, cutoff, schedule, batch, lda, ldb, ldc, stride_a, stride_b,
-                                                  stride_c, workspace_budget_bytes)
+                                                  stride_c, workspace_budget_bytes, flags)
         self._ws = None
 
     # -- introspection -------------------------------------------------------------

@@ -13,6 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libstrassen_b200.so")
 
 STRASSEN_OK = 0
+STRASSEN_FLAG_SINGLE_LEVEL_PASSES = 1
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SCHEDULE", -3: "WORKSPACE_TOO_SMALL", -4: "ALIAS",
                 -5: "MISALIGNED", -6: "CUDA_ERROR", -7: "OUT_OF_MEMORY"}
 K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_COUNT = range(7)
@@ -27,7 +28,7 @@ class strassen_options(ctypes.Structure):
     _fields_ = [("n", _i64), ("cutoff", _i64), ("schedule", _cp), ("batch", _i64),
                 ("lda", _i64), ("ldb", _i64), ("ldc", _i64),
                 ("stride_a", _i64), ("stride_b", _i64), ("stride_c", _i64),
-                ("workspace_budget_bytes", _sz)]
+                ("workspace_budget_bytes", _sz), ("flags", _i64)]
 
 
 SYMBOLS = [
@@ -99,9 +100,9 @@ def strassen_plan_create(n: int, cutoff: int, schedule) -> int:
 
 
 def strassen_plan_create_ex(n, cutoff, schedule=None, batch=1, lda=0, ldb=0, ldc=0, stride_a=0, stride_b=0,
-                            stride_c=0, workspace_budget_bytes=0) -> int:
+                            stride_c=0, workspace_budget_bytes=0, flags=0) -> int:
     o = strassen_options(n, cutoff, _sched(schedule), batch, lda, ldb, ldc, stride_a, stride_b, stride_c,
-                         workspace_budget_bytes)
+                         workspace_budget_bytes, flags)
     h = lib().strassen_plan_create_ex(ctypes.byref(o))
     if not h:
         raise StrassenError(-1, strassen_last_error())

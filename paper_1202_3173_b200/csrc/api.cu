@@ -54,6 +54,14 @@ struct strassen_plan {
 
 namespace {
 
+// Kernel family (strassen_kernel_kind) a launch is counted and timed under.
+int family(int op_kind)
+{
+    if (op_kind == OP_FORM2) return STRASSEN_K_FORM;
+    if (op_kind == OP_RECOMBINE2) return STRASSEN_K_RECOMBINE;
+    return op_kind;
+}
+
 int64_t extent_words(int64_t n, int64_t ld, int64_t stride, int64_t batch)
 {
     return (batch - 1) * stride + (n - 1) * ld + n;
@@ -151,6 +159,7 @@ strassen_plan *create(const strassen_options &o)
         delete p;
         return nullptr;
     }
+    d.fuse_two_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) == 0;
     d.sizes = level_sizes(n, cutoff);
     const size_t L = d.sizes.size() - 1;
     const bool want_auto = !o.schedule || strcmp(o.schedule, "auto") == 0;
@@ -204,7 +213,7 @@ strassen_plan *create(const strassen_options &o)
     }
     for (const Launch &op : d.launches) {
         const int k = launches_of(op);
-        p->launches[op.kind] += k;
+        p->launches[family(op.kind)] += k;
         p->launch_total += k;
     }
     return p;
@@ -257,7 +266,7 @@ int strassen_dgemm(strassen_plan *p, const double *A, const double *B, double *C
     int launched = 0;
     for (const Launch &op : d.launches) {
         const bool vec = op.vec_ok && bases16;
-        TimedLaunch t{op.kind, nullptr, nullptr};
+        TimedLaunch t{family(op.kind), nullptr, nullptr};
         if (p->timing) {
             t.start = take_event(p);
             t.stop = take_event(p);
@@ -271,6 +280,8 @@ int strassen_dgemm(strassen_plan *p, const double *A, const double *B, double *C
         case OP_FORM_ONE: e = launch_form_one(p->d_tab, op, bases, vec, stream, &launched); break;
         case OP_ACCUMULATE: e = launch_accumulate(p->d_tab, op, bases, vec, stream, &launched); break;
         case OP_PEEL: e = launch_peel(p->d_tab, op, bases, stream, &launched); break;
+        case OP_FORM2: e = launch_form2(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
         }
         if (p->timing) {
             cudaEventRecord(t.stop, stream);

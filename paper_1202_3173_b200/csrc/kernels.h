@@ -23,6 +23,9 @@ cudaError_t launch_form(const Node *tab, const Launch &op, const Bases &bases, b
                         int *launched);
 cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
                              int *launched);
+cudaError_t launch_form2(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream, int *launched);
+cudaError_t launch_recombine2(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
+                              int *launched);
 cudaError_t launch_form_one(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
                             int *launched);
 cudaError_t launch_accumulate(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,

@@ -54,6 +54,36 @@ struct Builder {
         return at;
     }
 
+    // The 7 children of each of the N nodes at p->nodes[tab ..) for a BFS step at level `lv`.
+    std::vector<Node> bfs_children(int64_t tab, int64_t N, const LevelInfo &lv) const
+    {
+        const int64_t h = lv.h, mat = lv.mat_words, ldw = lv.ldw;
+        std::vector<Node> kids(static_cast<size_t>(N) * 7, Node{});
+        const int64_t t_base = lv.ws_off, s_base = lv.ws_off + N * 4 * mat, q_base = lv.ws_off + N * 8 * mat;
+        for (int64_t q = 0; q < N; ++q) {
+            const Node nd = p->nodes[tab + q];
+            for (int j = 0; j < 7; ++j) {
+                Node &k = kids[size_t(q) * 7 + j];
+                k.a = kTQuad[j] >= 0 ? quadrant(nd.a, kTQuad[j], h) : ws_mat(t_base + (q * 4 + kTSlot[j]) * mat, ldw);
+                k.b = kSQuad[j] >= 0 ? quadrant(nd.b, kSQuad[j], h) : ws_mat(s_base + (q * 4 + kSSlot[j]) * mat, ldw);
+                k.c = ws_mat(q_base + (q * 7 + j) * mat, ldw);
+            }
+        }
+        return kids;
+    }
+
+    // Levels `level` and `level + 1` run as one two-level step when both are BFS steps, the lower
+    // one is not peeled (its fix-ups need the children's own products), and the run of BFS levels
+    // starting here has even length (so that the deepest levels, which move the most bytes, pair up).
+    bool pair_starts_here(int level) const
+    {
+        if (!p->fuse_two_levels) return false;
+        const int L = int(p->levels.size());
+        int run = 0;
+        while (level + run < L && p->levels[level + run].mode == 'B' && (run == 0 || !p->levels[level + run].peel)) ++run;
+        return run >= 2 && run % 2 == 0;
+    }
+
     // nodes of `level` are p->nodes[tab .. tab + count)
     void build(int level, int64_t tab, int64_t count)
     {
@@ -75,27 +105,39 @@ struct Builder {
             parents_even = parents_even && even(nd.a) && even(nd.b) && even(nd.c);
         }
         if (lv.mode == 'B') {
-            std::vector<Node> kids(static_cast<size_t>(N) * 7, Node{});
-            const int64_t t_base = lv.ws_off, s_base = lv.ws_off + N * 4 * mat, q_base = lv.ws_off + N * 8 * mat;
-            for (int64_t q = 0; q < N; ++q) {
-                const Node nd = p->nodes[tab + q];
-                for (int j = 0; j < 7; ++j) {
-                    Node &k = kids[size_t(q) * 7 + j];
-                    k.a = kTQuad[j] >= 0 ? quadrant(nd.a, kTQuad[j], h) : ws_mat(t_base + (q * 4 + kTSlot[j]) * mat, ldw);
-                    k.b = kSQuad[j] >= 0 ? quadrant(nd.b, kSQuad[j], h) : ws_mat(s_base + (q * 4 + kSSlot[j]) * mat, ldw);
-                    k.c = ws_mat(q_base + (q * 7 + j) * mat, ldw);
-                }
-            }
-            const int64_t ctab = append(kids);
+            const int64_t ctab = append(bfs_children(tab, N, lv));
             if (ctab < 0) return;
             Launch f{};
             f.kind = OP_FORM; f.level = level; f.j = -1; f.vec_ok = parents_even;
             f.parent_tab = tab; f.child_tab = ctab; f.count = N; f.m = lv.m; f.h = h;
-            p->launches.push_back(f);
-            build(level + 1, ctab, N * 7);
-            Launch r = f;
-            r.kind = OP_RECOMBINE;
-            p->launches.push_back(r);
+            f.grand_tab = -1;
+            if (pair_starts_here(level)) {
+                // two BFS levels in one pass: the children's sums are still written (the
+                // grandchildren's quadrant operands are views into them), their products are not
+                const LevelInfo &lv2 = p->levels[level + 1];
+                const int64_t gtab = append(bfs_children(ctab, N * 7, lv2));
+                if (gtab < 0) return;
+                f.kind = OP_FORM2;
+                f.grand_tab = gtab;
+                f.vec_ok = parents_even && (lv2.h & 1) == 0;
+                f.reg.child_t = lv.ws_off; f.reg.child_s = lv.ws_off + N * 4 * mat; f.reg.child_mat = mat;
+                f.reg.child_ld = int32_t(ldw);
+                const int64_t N2 = N * 7;
+                f.reg.grand_t = lv2.ws_off; f.reg.grand_s = lv2.ws_off + N2 * 4 * lv2.mat_words;
+                f.reg.grand_q = lv2.ws_off + N2 * 8 * lv2.mat_words; f.reg.grand_mat = lv2.mat_words;
+                f.reg.grand_ld = int32_t(lv2.ldw);
+                p->launches.push_back(f);
+                build(level + 2, gtab, N2 * 7);
+                Launch r = f;
+                r.kind = OP_RECOMBINE2;
+                p->launches.push_back(r);
+            } else {
+                p->launches.push_back(f);
+                build(level + 1, ctab, N * 7);
+                Launch r = f;
+                r.kind = OP_RECOMBINE;
+                p->launches.push_back(r);
+            }
         } else {
             const int64_t t_base = lv.ws_off, s_base = lv.ws_off + N * mat, q_base = lv.ws_off + 2 * N * mat;
             for (int j = 0; j < 7; ++j) {

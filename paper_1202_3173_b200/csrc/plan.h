@@ -32,7 +32,19 @@ enum OpKind : int32_t {
     OP_RECOMBINE = 2,  // BFS: 7 Q of each parent -> its four C quadrants
     OP_FORM_ONE = 3,   // DFS: operands of child j of each parent
     OP_ACCUMULATE = 4, // DFS: fold Q_j of each parent into its C quadrants
-    OP_PEEL = 5        // odd m: rank-one update, last column, last row
+    OP_PEEL = 5,       // odd m: rank-one update, last column, last row
+    OP_FORM2 = 6,      // two BFS levels at once: sums of the children and of the grandchildren
+    OP_RECOMBINE2 = 7  // two BFS levels at once: 49 grandchild products -> the parent's C
+};
+
+// Regular layout of the workspace regions a two-level launch writes / reads (element offsets
+// from the workspace base; slot s of child c sits at base + (c * slots + s) * mat).
+struct Regions2 {
+    int64_t child_t, child_s;            // level i+1 operand sums: 4 per parent and side
+    int64_t child_mat;
+    int64_t grand_t, grand_s, grand_q;   // level i+2: 4 + 4 sums and 7 products per child
+    int64_t grand_mat;
+    int32_t child_ld, grand_ld;
 };
 
 struct Launch {
@@ -46,6 +58,8 @@ struct Launch {
     int64_t count;       // number of parents (leaves)
     int64_t m;           // size of the parents (leaves)
     int64_t h;           // size of the children
+    int64_t grand_tab;   // OP_FORM2 / OP_RECOMBINE2: index of the first grandchild node
+    Regions2 reg;        // OP_FORM2 / OP_RECOMBINE2 only
 };
 
 struct LevelInfo {
@@ -63,6 +77,7 @@ struct PlanDesc {
     int64_t n = 0, cutoff = 0, batch = 1;
     int64_t lda = 0, ldb = 0, ldc = 0;
     int64_t stride_a = 0, stride_b = 0, stride_c = 0;
+    bool fuse_two_levels = true;    // run pairs of consecutive BFS levels as OP_FORM2 / OP_RECOMBINE2
     std::string schedule;           // resolved, one char per level
     std::vector<int64_t> sizes;     // m_0 .. m_L
     std::vector<LevelInfo> levels;  // L entries

@@ -109,6 +109,26 @@ def test_inputs_are_not_written_and_calls_repeat():
     assert torch.equal(C1, C2)          # same plan, same inputs: same bits
 
 
+@pytest.mark.parametrize("n,cutoff,sched,dist", [(1024, 128, "BBB", "uniform"), (1024, 256, "BB", "normal"),
+                                                 (512, 32, "BBBB", "uniform"), (520, 65, "BBB", "uniform"),
+                                                 (1030, 64, "BDBB", "uniform"), (771, 96, "BBB", "uniform"),
+                                                 (197, 12, "BBBB", "uniform"), (36, 9, "BB", "int8"),
+                                                 (1544, 193, "DBB", "normal")])
+def test_two_level_passes_give_the_same_bits_as_single_level_passes(n, cutoff, sched, dist):
+    A, B = inputs.pair(n, dist, n + 7, device="cuda")
+    fused = run_plan(n, cutoff, sched, A, B)
+    single = run_plan(n, cutoff, sched, A, B, flags=binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
+    assert torch.equal(fused, single)      # same operations in the same order
+    p1, p2 = Plan(n, cutoff, sched), Plan(n, cutoff, sched, flags=binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
+    assert p1.launch_count <= p2.launch_count
+    p1.close(); p2.close()
+
+
+def test_batch_with_two_level_passes():
+    check_full(256, 64, "BB", "uniform", 121, batch=6)
+    check_full(260, 65, "BB", "int8", 122, batch=3)      # odd quarter size: 8-byte accesses
+
+
 def test_schedules_agree_exactly_on_integers():
     A, B = inputs.pair(512, "int8", 41, device="cuda")
     outs = [run_plan(512, 64, s, A, B) for s in ("BBB", "DDD", "BDB", "DBD")]

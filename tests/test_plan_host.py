@@ -126,16 +126,30 @@ def test_auto_without_budget_or_device_fails_loudly():
 
 
 def test_launch_lists():
-    # all BFS: one form and one recombine per level, one batched product launch
-    p = Plan(4096, 512, "BBB")
+    # all BFS, one pass per level: one form and one recombine per level, one batched product launch
+    single = binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES
+    p = Plan(4096, 512, "BBB", flags=single)
     assert p.launches_by_kind() == {"form": 3, "gemm": 1, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0}
     assert p.launch_count == 7
     p.close()
+    # default: the two deepest BFS levels share one formation pass and one recombination pass
+    p = Plan(4096, 512, "BBB")
+    assert p.launches_by_kind() == {"form": 2, "gemm": 1, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0}
+    p.close()
     # DFS on top: 7 x (form_one [not for j = 0, 1], sub-tree, accumulate)
-    p = Plan(16384, 512, "DBBBB")
+    p = Plan(16384, 512, "DBBBB", flags=single)
     k = p.launches_by_kind()
     assert k["form_one"] == 5 and k["accumulate"] == 7 and k["gemm"] == 7 and k["form"] == 28 and k["recombine"] == 28
     assert p.base_products == 7 ** 5
+    p.close()
+    p = Plan(16384, 512, "DBBBB")          # four BFS levels below the DFS step: two pairs
+    k = p.launches_by_kind()
+    assert k["form"] == 14 and k["recombine"] == 14 and k["gemm"] == 7 and p.base_products == 7 ** 5
+    p.close()
+    # a peeled level cannot be the lower half of a pair (its fix-ups need the children's products)
+    p = Plan(12345, 771, "BBBB")           # sizes 12345, 6172, 3086, 1543 (odd), 771: pairs (0,1) and none at (2,3)
+    k = p.launches_by_kind()
+    assert k["form"] == 3 and k["recombine"] == 3
     p.close()
     # all DFS: 7^L single products
     p = Plan(64, 8, "DDD")
