@@ -412,75 +412,111 @@ __global__ void __launch_bounds__(256) peel_rank1_kernel(const Node *__restrict_
     }
 }
 
-constexpr int PC_ROWS = 32, PC_CHUNK = 1024;
-__global__ void __launch_bounds__(256) peel_col_kernel(const Node *__restrict__ nodes, Bases bases, int m, int item0)
+// Thin products: a few columns or a few rows of C = A.B of one node, over the full inner
+// dimension K.  They serve the peeled last column / row (one of each) and the ragged remainder of
+// base products whose size is a few elements past a multiple of the GEMM tile (e.g. 771 = 768 + 3).
+// Both read one operand in full once; summation order is fixed (bit-reproducible).
+
+// Columns [c0, c0 + nc) of C for rows [0, rows): each warp owns 4 rows, lanes stride over k; the nc
+// columns of B are staged through shared memory in chunks of TC_CHUNK rows.
+constexpr int TC_ROWS = 32, TC_CHUNK = 512;
+template <int NC>
+__global__ void __launch_bounds__(256) thin_cols_kernel(const Node *__restrict__ nodes, Bases bases, int K, int rows,
+                                                        int c0, int nc, int item0)
 {
-    __shared__ double bcol[PC_CHUNK];
+    __shared__ double bs[NC][TC_CHUNK];
     const Node nd = nodes[item0 + blockIdx.y];
     const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
     double *C = resolve(bases, nd.c);
-    const int e = m - 1, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rbase = blockIdx.x * PC_ROWS + warp * 4;
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
-    for (int k0 = 0; k0 < m; k0 += PC_CHUNK) {
-        const int kn = min(PC_CHUNK, m - k0);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rbase = blockIdx.x * TC_ROWS + warp * 4;
+    double acc[4][NC];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int t = 0; t < NC; ++t) acc[i][t] = 0.0;
+    for (int k0 = 0; k0 < K; k0 += TC_CHUNK) {
+        const int kn = min(TC_CHUNK, K - k0);
         __syncthreads();
-        for (int k = threadIdx.x; k < kn; k += 256) bcol[k] = B[int64_t(k0 + k) * nd.b.ld + e];
+        for (int e = threadIdx.x; e < kn * NC; e += 256) {
+            const int k = e / NC, t = e % NC;
+            bs[t][k] = t < nc ? B[int64_t(k0 + k) * nd.b.ld + c0 + t] : 0.0;
+        }
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int r = rbase + i;
-            if (r < m) {
+            if (r < rows) {
                 const double *a = A + int64_t(r) * nd.a.ld + k0;
-                double s = acc[i];
-                for (int k = lane; k < kn; k += 32) s = fma(a[k], bcol[k], s);
-                acc[i] = s;
+                for (int k = lane; k < kn; k += 32) {
+                    const double av = a[k];
+#pragma unroll
+                    for (int t = 0; t < NC; ++t) acc[i][t] = fma(av, bs[t][k], acc[i][t]);
+                }
             }
         }
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        double s = acc[i];
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
         const int r = rbase + i;
-        if (lane == 0 && r < m) C[int64_t(r) * nd.c.ld + e] = s;
+#pragma unroll
+        for (int t = 0; t < NC; ++t) {
+            double v = acc[i][t];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+            if (lane == 0 && r < rows && t < nc) C[int64_t(r) * nd.c.ld + c0 + t] = v;
+        }
     }
 }
 
-constexpr int PR_COLS = 32, PR_SLICES = 16;
-__global__ void __launch_bounds__(PR_COLS *PR_SLICES) peel_row_kernel(const Node *__restrict__ nodes, Bases bases,
-                                                                      int m, int item0)
+// Rows [r0, r0 + nr) of C for columns [0, cols): a thread owns one column and every TR_SLICES-th k;
+// the slices are summed through shared memory in a fixed order.
+constexpr int TR_COLS = 32, TR_SLICES = 16;
+template <int NR>
+__global__ void __launch_bounds__(TR_COLS *TR_SLICES) thin_rows_kernel(const Node *__restrict__ nodes, Bases bases, int K,
+                                                                      int cols, int r0, int nr, int item0)
 {
-    __shared__ double part[PR_SLICES][PR_COLS + 1];
+    __shared__ double part[TR_SLICES][NR][TR_COLS + 1];
     const Node nd = nodes[item0 + blockIdx.y];
     const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
     double *C = resolve(bases, nd.c);
-    const int e = m - 1;
-    const int c = blockIdx.x * PR_COLS + threadIdx.x;
-    const double *arow = A + int64_t(e) * nd.a.ld;
-    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-    if (c < e) {
-        const double *b = B + c;
-        const int64_t ldb = nd.b.ld;
-        int k = threadIdx.y;
-        for (; k + 3 * PR_SLICES < m; k += 4 * PR_SLICES) {
-            const double b0 = b[int64_t(k) * ldb], b1 = b[int64_t(k + PR_SLICES) * ldb];
-            const double b2 = b[int64_t(k + 2 * PR_SLICES) * ldb], b3 = b[int64_t(k + 3 * PR_SLICES) * ldb];
-            s0 = fma(arow[k], b0, s0);
-            s1 = fma(arow[k + PR_SLICES], b1, s1);
-            s2 = fma(arow[k + 2 * PR_SLICES], b2, s2);
-            s3 = fma(arow[k + 3 * PR_SLICES], b3, s3);
-        }
-        for (; k < m; k += PR_SLICES) s0 = fma(arow[k], b[int64_t(k) * ldb], s0);
-    }
-    part[threadIdx.y][threadIdx.x] = (s0 + s1) + (s2 + s3);
-    __syncthreads();
-    if (threadIdx.y == 0 && c < e) {
-        double s = 0.0;
+    const int c = blockIdx.x * TR_COLS + threadIdx.x;
+    double acc[NR];
 #pragma unroll
-        for (int i = 0; i < PR_SLICES; ++i) s += part[i][threadIdx.x];
-        C[int64_t(e) * nd.c.ld + c] = s;
+    for (int t = 0; t < NR; ++t) acc[t] = 0.0;
+    if (c < cols) {
+        const double *b = B + c;
+        const int64_t ldb = nd.b.ld, lda = nd.a.ld;
+        const double *arow = A + int64_t(r0) * lda;
+        int k = threadIdx.y;
+        for (; k + 3 * TR_SLICES < K; k += 4 * TR_SLICES) {
+            double bv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) bv[u] = b[int64_t(k + u * TR_SLICES) * ldb];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int t = 0; t < NR; ++t)
+                    if (t < nr) acc[t] = fma(arow[int64_t(t) * lda + k + u * TR_SLICES], bv[u], acc[t]);
+        }
+        for (; k < K; k += TR_SLICES) {
+            const double bv = b[int64_t(k) * ldb];
+#pragma unroll
+            for (int t = 0; t < NR; ++t)
+                if (t < nr) acc[t] = fma(arow[int64_t(t) * lda + k], bv, acc[t]);
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < NR; ++t) part[threadIdx.y][t][threadIdx.x] = acc[t];
+    __syncthreads();
+    if (threadIdx.y == 0 && c < cols) {
+#pragma unroll
+        for (int t = 0; t < NR; ++t) {
+            double v = 0.0;
+#pragma unroll
+            for (int i = 0; i < TR_SLICES; ++i) v += part[i][t][threadIdx.x];
+            if (t < nr) C[int64_t(r0 + t) * nd.c.ld + c] = v;
+        }
     }
 }
 
@@ -501,7 +537,10 @@ int launches_of(const Launch &op)
     case OP_FORM_ONE: return chunks(op.count * ((op.j >= 2 && op.j <= 4) ? 2 : 1));
     case OP_ACCUMULATE: return chunks(op.count);
     case OP_PEEL: return 3 * chunks(op.count);
-    case OP_GEMM: return 1;
+    case OP_GEMM: {
+        const int rem = gemm_thin_remainder(op.m), bulk = int(op.m) - rem;
+        return (bulk > 0 ? 1 : 0) + (rem ? chunks(op.count) * (bulk > 0 ? 2 : 1) : 0);
+    }
     case OP_FORM2: return chunks(op.count * 2);
     case OP_RECOMBINE2: return chunks(op.count);
     }
@@ -614,21 +653,49 @@ cudaError_t launch_accumulate(const Node *tab, const Launch &op, const Bases &ba
     return cudaGetLastError();
 }
 
+cudaError_t launch_thin_cols(const Node *nodes, const Bases &bases, int K, int rows, int c0, int nc, int64_t count,
+                             cudaStream_t stream, int *launched)
+{
+    const int64_t total = count;
+    FOR_CHUNKS(total) {
+        const dim3 grid((rows + TC_ROWS - 1) / TC_ROWS, unsigned(zn));
+        if (nc <= 1) thin_cols_kernel<1><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        else if (nc <= 2) thin_cols_kernel<2><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        else if (nc <= 4) thin_cols_kernel<4><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        else thin_cols_kernel<8><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int cols, int r0, int nr, int64_t count,
+                             cudaStream_t stream, int *launched)
+{
+    const int64_t total = count;
+    FOR_CHUNKS(total) {
+        const dim3 grid((cols + TR_COLS - 1) / TR_COLS, unsigned(zn)), block(TR_COLS, TR_SLICES);
+        if (nr <= 1) thin_rows_kernel<1><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+        else if (nr <= 2) thin_rows_kernel<2><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+        else if (nr <= 4) thin_rows_kernel<4><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+        else thin_rows_kernel<8><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
 cudaError_t launch_peel(const Node *tab, const Launch &op, const Bases &bases, cudaStream_t stream, int *launched)
 {
     const int m = int(op.m), e = m - 1;
+    const Node *nodes = tab + op.parent_tab;
     const int64_t total = op.count;
     FOR_CHUNKS(total) {
-        const Node *nodes = tab + op.parent_tab;
         peel_rank1_kernel<<<dim3((e + 63) / 64, (e + TILE_ROWS - 1) / TILE_ROWS, unsigned(zn)), dim3(64, TY), 0,
                             stream>>>(nodes, bases, e, int(item0));
-        peel_col_kernel<<<dim3((m + PC_ROWS - 1) / PC_ROWS, unsigned(zn)), 256, 0, stream>>>(nodes, bases, m,
-                                                                                             int(item0));
-        peel_row_kernel<<<dim3((e + PR_COLS - 1) / PR_COLS, unsigned(zn)), dim3(PR_COLS, PR_SLICES), 0, stream>>>(
-            nodes, bases, m, int(item0));
-        *launched += 3;
+        ++*launched;
     }
-    return cudaGetLastError();
+    cudaError_t err = launch_thin_cols(nodes, bases, m, m, e, 1, op.count, stream, launched);   // last column, all rows
+    if (err != cudaSuccess) return err;
+    return launch_thin_rows(nodes, bases, m, e, e, 1, op.count, stream, launched);              // last row, other columns
 }
 
 }  // namespace strassen

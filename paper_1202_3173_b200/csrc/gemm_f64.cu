@@ -20,21 +20,18 @@
 //     (size not a multiple of 128 / 16) are zero-filled by cp.async's src-size operand and
 //     masked in the epilogue; operands that are only 8-byte aligned (views into matrices
 //     with an odd leading dimension) use 8-byte copies.
-#include <cstdlib>
-
 #include "kernels.h"
 
 namespace strassen {
 
 namespace {
 
-constexpr int BM = 128;
-
-// Tile shape variants: BN columns per CTA tile (each warp owns 64 x 32, warps are 2 x BN/32),
+// Tile shape variants: BM x BN CTA tile, each warp owns WTM x 32 of it (warps are BM/WTM x BN/32),
 // BK-deep slabs, STAGES slabs in the ring, CTAS resident per SM.
-template <int BN_, int BK_, int STAGES_, int CTAS_> struct Cfg {
-    static constexpr int BN = BN_, BK = BK_, STAGES = STAGES_, CTAS = CTAS_;
-    static constexpr int WARPS_N = BN / 32, THREADS = 2 * WARPS_N * 32;
+template <int BM_, int BN_, int WTM_, int BK_, int STAGES_, int CTAS_> struct Cfg {
+    static constexpr int BM = BM_, BN = BN_, WTM = WTM_, BK = BK_, STAGES = STAGES_, CTAS = CTAS_;
+    static constexpr int WARPS_N = BN / 32, THREADS = (BM / WTM) * WARPS_N * 32;
+    static constexpr int MT = WTM / 8;                // DMMA accumulator tiles along m per warp
     static constexpr int AS = BK + 4;                 // padded row of the A slab (doubles)
     static constexpr int BS = BN + 4;                 // padded row of the B slab
     static constexpr int A_STAGE = BM * AS, B_STAGE = BK * BS;
@@ -47,9 +44,11 @@ template <int BN_, int BK_, int STAGES_, int CTAS_> struct Cfg {
     static constexpr int B_CHUNKS = BK / B_KROWS_STEP;          // passes for the B slab
     static_assert(BK % 8 == 0 && AS % 16 == 4 && BS % 16 == 4, "fragment loads rely on stride = 4 mod 16");
 };
-using CfgWide = Cfg<128, 16, 4, 1>;     // 149.5 KB of shared memory, one CTA per SM
-using CfgPair = Cfg<64, 16, 3, 2>;      // 87.6 KB, two independent CTAs per SM
-using CfgDeep = Cfg<128, 32, 3, 1>;     // 212 KB: half as many barriers per tile
+// Measured alternatives that did not beat CfgWide on 343 x 512^3 (33.9 TFLOP/s): 128 x 64 tiles with two
+// CTAs per SM (32.7), 32-deep slabs (33.9), 64 x 128 tiles with 16 warps per SM (33.9).
+using CfgWide = Cfg<128, 128, 64, 16, 4, 1>;    // 8 warps of 64 x 32; 149.5 KB of shared memory, one CTA per SM
+using CfgSmall = Cfg<64, 64, 32, 16, 4, 2>;     // 4 warps of 32 x 32; 54 KB: four times as many tiles, for launches
+                                                // whose 128 x 128 tiles would leave most SMs idle
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
 {
@@ -79,7 +78,7 @@ struct TileCoord {
     int node, m0, n0;
 };
 
-template <int BN>
+template <int BM, int BN>
 __device__ __forceinline__ TileCoord tile_coord(long long t, int tiles_n, int tiles_per_node)
 {
     TileCoord c;
@@ -104,10 +103,11 @@ struct LoadState {
 
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, C::CTAS)
-gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n, int tiles_per_node, int ktiles,
+gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int tiles_n, int tiles_per_node, int ktiles,
                 long long total_tiles)
 {
-    constexpr int BN = C::BN, BK = C::BK, AS = C::AS, BS = C::BS, STAGES = C::STAGES, STAGE_WORDS = C::STAGE_WORDS;
+    // M: extent of the output block computed here (rows and columns); K: inner dimension.
+    constexpr int BM = C::BM, BN = C::BN, WTM = C::WTM, MT = C::MT, BK = C::BK, AS = C::AS, BS = C::BS, STAGES = C::STAGES, STAGE_WORDS = C::STAGE_WORDS;
     constexpr int A_STAGE = C::A_STAGE, A_CHUNKS = C::A_CHUNKS, A_ROWS_STEP = C::A_ROWS_STEP, A_KCHUNKS = C::A_KCHUNKS;
     constexpr int B_CHUNKS = C::B_CHUNKS, B_KROWS_STEP = C::B_KROWS_STEP;
     extern __shared__ __align__(16) double smem[];
@@ -122,7 +122,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
     const int b_krow0 = tid / (BN / 2), b_nc = tid % (BN / 2);
     const uint32_t a_dst0 = smem_base + uint32_t((a_row0 * AS + a_kc * 2) * 8);
     const uint32_t b_dst0 = smem_base + uint32_t((A_STAGE + b_krow0 * BS + b_nc * 2) * 8);
-    const bool k_ragged = (M % BK) != 0;
+    const bool k_ragged = (K % BK) != 0;
 
     long long load_tile = blockIdx.x;
     int load_k = 0;
@@ -131,7 +131,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
 
     // The node of the tile whose loads start next is fetched one slab ahead of its use, so that
     // the table read never sits between a warp and its next DMMAs.
-    TileCoord next_tc = tile_coord<BN>(load_tile < total_tiles ? load_tile : 0, tiles_n, tiles_per_node);
+    TileCoord next_tc = tile_coord<BM, BN>(load_tile < total_tiles ? load_tile : 0, tiles_n, tiles_per_node);
     Operand next_a = nodes[next_tc.node].a, next_b = nodes[next_tc.node].b;
 
     auto setup_load = [&]() {
@@ -169,8 +169,8 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                     cp_async16_full(b_dst0 + soff + uint32_t(B_KROWS_STEP * i * BS * 8), ls.b + i * ls.b_step);
             } else {
                 const int k0 = load_k * BK;
-                // A slab: 128 rows x 16 k (K == M: the leaves are square)
-                const int kvalid = max(0, min(2, M - (k0 + a_kc * 2)));
+                // A slab: BM rows x BK k
+                const int kvalid = max(0, min(2, K - (k0 + a_kc * 2)));
 #pragma unroll
                 for (int i = 0; i < A_CHUNKS; ++i) {
                     const int nv = ((ls.a_rows_ok >> i) & 1) ? kvalid : 0;
@@ -186,7 +186,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                 // B slab: 16 k x 128 columns
 #pragma unroll
                 for (int i = 0; i < B_CHUNKS; ++i) {
-                    const int nv = (k0 + b_krow0 + B_KROWS_STEP * i) < M ? ls.b_cols : 0;
+                    const int nv = (k0 + b_krow0 + B_KROWS_STEP * i) < K ? ls.b_cols : 0;
                     const double *s = nv ? ls.b + i * ls.b_step : safe;
                     const uint32_t dst = b_dst0 + soff + uint32_t(B_KROWS_STEP * i * BS * 8);
                     if (ls.b16) {
@@ -203,7 +203,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
                 load_k = 0;
                 load_tile += gridDim.x;
                 if (load_tile < total_tiles) {
-                    next_tc = tile_coord<BN>(load_tile, tiles_n, tiles_per_node);
+                    next_tc = tile_coord<BM, BN>(load_tile, tiles_n, tiles_per_node);
                     next_a = nodes[next_tc.node].a;
                     next_b = nodes[next_tc.node].b;
                 }
@@ -212,26 +212,26 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
         cp_async_commit();
     };
 
-    double acc[8][4][2];
+    double acc[MT][4][2];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < MT; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
 
     // fragments of one 4-deep step: A[64 rows of the warp][4 k] and B[4 k][32 columns of the warp]
-    const double *a_frag0 = smem + (wm * 64 + g) * AS + q;
+    const double *a_frag0 = smem + (wm * WTM + g) * AS + q;
     const double *b_frag0 = smem + A_STAGE + q * BS + wn * 32 + g;
-    auto load_frags = [&](int slot, int kk, double (&fa)[8], double (&fb)[4]) {
+    auto load_frags = [&](int slot, int kk, double (&fa)[MT], double (&fb)[4]) {
         const double *As = a_frag0 + slot * STAGE_WORDS + kk * 4;
         const double *Bs = b_frag0 + slot * STAGE_WORDS + kk * 4 * BS;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) fa[i] = As[i * 8 * AS];
+        for (int i = 0; i < MT; ++i) fa[i] = As[i * 8 * AS];
 #pragma unroll
         for (int j = 0; j < 4; ++j) fb[j] = Bs[j * 8];
     };
-    auto mma_step = [&](const double (&fa)[8], const double (&fb)[4]) {
+    auto mma_step = [&](const double (&fa)[MT], const double (&fb)[4]) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < MT; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) dmma(acc[i][j][0], acc[i][j][1], fa[i], fb[j]);
     };
@@ -241,12 +241,12 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
     cp_async_wait<STAGES - 2>();      // slab 0 has landed
     __syncthreads();
 
-    double fa0[8], fb0[4], fa1[8], fb1[4];
+    double fa0[MT], fb0[4], fa1[MT], fb1[4];
     int slot = 0;
     load_frags(slot, 0, fa0, fb0);
 
     for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const TileCoord tc = tile_coord<BN>(tile, tiles_n, tiles_per_node);
+        const TileCoord tc = tile_coord<BM, BN>(tile, tiles_n, tiles_per_node);
         const Operand c_op = nodes[tc.node].c;        // consumed after the k loop
         for (int kt = 0; kt < ktiles; ++kt) {
             // Invariant: every warp has passed the barrier of the previous slab, i.e. has finished
@@ -271,12 +271,12 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
         double *C = base_ptr(bases, c_op.base) + c_op.off;
         const long long ldc = c_op.ld;
         const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((c_op.ld & 1) == 0);
-        const int r0 = tc.m0 + wm * 64 + g, c0 = tc.n0 + wn * 32 + q * 2;
+        const int r0 = tc.m0 + wm * WTM + g, c0 = tc.n0 + wn * 32 + q * 2;
         double *o = C + (long long)r0 * ldc + c0;
         if (c16 && tc.m0 + BM <= M && tc.n0 + BN <= M) {
             // interior tile: 16-byte stores at fixed offsets from one running row pointer
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < MT; ++i) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     *reinterpret_cast<double2 *>(o + j * 8) = make_double2(acc[i][j][0], acc[i][j][1]);
@@ -286,7 +286,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < MT; ++i) {
                 const int r = r0 + i * 8;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -313,7 +313,8 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int tiles_n,
 namespace {
 
 template <class C>
-cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, long long count, int sm_count, cudaStream_t stream)
+cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, int K, long long count, int sm_count,
+                       cudaStream_t stream)
 {
     static bool configured[64] = {false};   // per device: opt in to > 48 KB of dynamic shared memory
     int dev = 0;
@@ -324,13 +325,13 @@ cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, long long c
         if (e != cudaSuccess) return e;
         if (dev < 64) configured[dev] = true;
     }
-    const int tiles_m = (M + BM - 1) / BM, tiles_n = (M + C::BN - 1) / C::BN;
+    const int tiles_m = (M + C::BM - 1) / C::BM, tiles_n = (M + C::BN - 1) / C::BN;
     const int tiles_per_node = tiles_m * tiles_n;
-    const int ktiles = (M + C::BK - 1) / C::BK;
+    const int ktiles = (K + C::BK - 1) / C::BK;
     const long long total = (long long)tiles_per_node * count;
     const long long slots = (long long)sm_count * C::CTAS;
     const int grid = int(total < slots ? total : slots);
-    gemm_f64_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(nodes, bases, M, tiles_n, tiles_per_node, ktiles, total);
+    gemm_f64_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(nodes, bases, M, K, tiles_n, tiles_per_node, ktiles, total);
     return cudaGetLastError();
 }
 
@@ -339,14 +340,31 @@ cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, long long c
 cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
                         int *launched)
 {
-    static const int variant = [] {
-        const char *v = getenv("STRASSEN_GEMM_VARIANT");
-        return v ? atoi(v) : 0;
-    }();
-    ++*launched;
-    if (variant == 1) return launch_cfg<CfgPair>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
-    if (variant == 2) return launch_cfg<CfgDeep>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
-    return launch_cfg<CfgWide>(tab + op.parent_tab, bases, int(op.m), op.count, sm_count, stream);
+    // A size a few elements past a multiple of 64 would spend a whole extra row and column of tiles on
+    // those elements: the tiles cover the multiple, thin products the remainder.
+    const int K = int(op.m), rem = gemm_thin_remainder(op.m), M = K - rem;
+    const Node *nodes = tab + op.parent_tab;
+    cudaError_t err = cudaSuccess;
+    if (M > 0) {
+        ++*launched;
+        // Few large tiles leave SMs idle: when the 128 x 128 tiling cannot give every SM a tile, the 64 x 64
+        // tiling (two CTAs per SM) is compared by rounds x tile cost (a 128 x 128 tile = 8 units).
+        const long long t_wide = (long long)((M + 127) / 128) * ((M + 127) / 128) * op.count;
+        const long long t_small = (long long)((M + 63) / 64) * ((M + 63) / 64) * op.count;
+        const long long cost_wide = ((t_wide + sm_count - 1) / sm_count) * 8;
+        const long long cost_small = t_small <= sm_count ? 2 : ((t_small + 2 * sm_count - 1) / (2 * sm_count)) * 4 + 1;
+        if (cost_small * 10 < cost_wide * 9)
+            err = launch_cfg<CfgSmall>(nodes, bases, M, K, op.count, sm_count, stream);
+        else
+            err = launch_cfg<CfgWide>(nodes, bases, M, K, op.count, sm_count, stream);
+        if (err != cudaSuccess) return err;
+    }
+    if (rem) {
+        err = launch_thin_cols(nodes, bases, K, K, M, rem, op.count, stream, launched);     // columns [M, K), all rows
+        if (err != cudaSuccess) return err;
+        if (M > 0) err = launch_thin_rows(nodes, bases, K, M, M, rem, op.count, stream, launched);   // rows [M, K), columns [0, M)
+    }
+    return err;
 }
 
 }  // namespace strassen

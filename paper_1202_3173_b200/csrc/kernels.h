@@ -34,6 +34,21 @@ cudaError_t launch_peel(const Node *tab, const Launch &op, const Bases &bases, c
 cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
                         int *launched);
 
+// Thin products over `count` nodes (full inner dimension K): columns [c0, c0 + nc) for rows [0, rows),
+// and rows [r0, r0 + nr) for columns [0, cols); nc, nr <= 8.
+cudaError_t launch_thin_cols(const Node *nodes, const Bases &bases, int K, int rows, int c0, int nc, int64_t count,
+                             cudaStream_t stream, int *launched);
+cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int cols, int r0, int nr, int64_t count,
+                             cudaStream_t stream, int *launched);
+
+// A base product whose size is 1..8 past a multiple of 64 is computed as a tiled bulk of that
+// multiple plus thin products for the remainder rows / columns; returns the remainder (0 = none).
+inline int gemm_thin_remainder(int64_t m)
+{
+    const int rem = int(m % 64);
+    return rem >= 1 && rem <= 8 ? rem : 0;
+}
+
 // Kernels one replay of `op` launches (host arithmetic only; mirrors the launchers).
 int launches_of(const Launch &op);
 
