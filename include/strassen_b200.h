@@ -154,7 +154,8 @@ int strassen_plan_levels(const strassen_plan *plan);                    /* L    
 int64_t strassen_plan_level_size(const strassen_plan *plan, int level); /* m_level, 0 <= level <= L  */
 int64_t strassen_plan_base_size(const strassen_plan *plan);             /* m_L                        */
 int64_t strassen_plan_base_products(const strassen_plan *plan);         /* batch * 7^L                */
-int64_t strassen_plan_launch_count(const strassen_plan *plan);          /* kernels per strassen_dgemm */
+int64_t strassen_plan_launch_count(const strassen_plan *plan);          /* kernels per strassen_dgemm (counted
+                                                                           for a 148-SM device)       */
 int64_t strassen_plan_launches_of(const strassen_plan *plan, int kind); /* ... of one family          */
 
 /* Workspace (bytes, unpadded) a schedule string needs under the paper's accounting of 21

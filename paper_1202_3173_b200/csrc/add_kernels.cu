@@ -539,7 +539,12 @@ int launches_of(const Launch &op)
     case OP_PEEL: return 3 * chunks(op.count);
     case OP_GEMM: {
         const int rem = gemm_thin_remainder(op.m), bulk = int(op.m) - rem;
-        return (bulk > 0 ? 1 : 0) + (rem ? chunks(op.count) * (bulk > 0 ? 2 : 1) : 0);
+        int tiled = 0;
+        if (bulk > 0) {
+            const GemmSplit split = gemm_split(bulk, op.count, kNominalSMs);
+            tiled = (!split.all_small && split.wide_leaves < op.count) ? 2 : 1;
+        }
+        return tiled + (rem ? chunks(op.count) * (bulk > 0 ? 2 : 1) : 0);
     }
     case OP_FORM2: return chunks(op.count * 2);
     case OP_RECOMBINE2: return chunks(op.count);

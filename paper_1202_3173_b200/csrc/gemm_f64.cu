@@ -42,10 +42,11 @@ template <int BM_, int BN_, int WTM_, int BK_, int STAGES_, int CTAS_> struct Cf
     static constexpr int A_CHUNKS = BM / A_ROWS_STEP;           // passes (chunks per thread) for the A slab
     static constexpr int B_KROWS_STEP = THREADS / (BN / 2);     // B rows covered by one pass
     static constexpr int B_CHUNKS = BK / B_KROWS_STEP;          // passes for the B slab
-    static_assert(BK % 8 == 0 && AS % 16 == 4 && BS % 16 == 4, "fragment loads rely on stride = 4 mod 16");
+    static_assert(BK % 8 == 0 && (AS % 16 == 4 || AS % 16 == 12) && BS % 16 == 4, "fragment loads rely on these strides");
 };
 // Measured alternatives that did not beat CfgWide on 343 x 512^3 (33.9 TFLOP/s): 128 x 64 tiles with two
-// CTAs per SM (32.7), 32-deep slabs (33.9), 64 x 128 tiles with 16 warps per SM (33.9).
+// CTAs per SM (32.7), 32-deep slabs (33.9), 8-deep slabs (32.7), 64 x 128 tiles with 16 warps per SM (33.9).
+// What remains per tile is the drain of its 128 KB of stores (about 2.4 us of a 71 us tile at K = 512).
 using CfgWide = Cfg<128, 128, 64, 16, 4, 1>;    // 8 warps of 64 x 32; 149.5 KB of shared memory, one CTA per SM
 using CfgSmall = Cfg<64, 64, 32, 16, 4, 2>;     // 4 warps of 32 x 32; 54 KB: four times as many tiles, for launches
                                                 // whose 128 x 128 tiles would leave most SMs idle
@@ -346,17 +347,19 @@ cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, i
     const Node *nodes = tab + op.parent_tab;
     cudaError_t err = cudaSuccess;
     if (M > 0) {
-        ++*launched;
-        // Few large tiles leave SMs idle: when the 128 x 128 tiling cannot give every SM a tile, the 64 x 64
-        // tiling (two CTAs per SM) is compared by rounds x tile cost (a 128 x 128 tile = 8 units).
-        const long long t_wide = (long long)((M + 127) / 128) * ((M + 127) / 128) * op.count;
-        const long long t_small = (long long)((M + 63) / 64) * ((M + 63) / 64) * op.count;
-        const long long cost_wide = ((t_wide + sm_count - 1) / sm_count) * 8;
-        const long long cost_small = t_small <= sm_count ? 2 : ((t_small + 2 * sm_count - 1) / (2 * sm_count)) * 4 + 1;
-        if (cost_small * 10 < cost_wide * 9)
+        const GemmSplit split = gemm_split(M, op.count, sm_count);
+        if (split.all_small) {
+            ++*launched;
             err = launch_cfg<CfgSmall>(nodes, bases, M, K, op.count, sm_count, stream);
-        else
-            err = launch_cfg<CfgWide>(nodes, bases, M, K, op.count, sm_count, stream);
+        } else {
+            ++*launched;
+            err = launch_cfg<CfgWide>(nodes, bases, M, K, split.wide_leaves, sm_count, stream);
+            if (err == cudaSuccess && split.wide_leaves < op.count) {
+                ++*launched;
+                err = launch_cfg<CfgSmall>(nodes + split.wide_leaves, bases, M, K, op.count - split.wide_leaves, sm_count,
+                                           stream);
+            }
+        }
         if (err != cudaSuccess) return err;
     }
     if (rem) {

@@ -49,6 +49,35 @@ inline int gemm_thin_remainder(int64_t m)
     return rem >= 1 && rem <= 8 ? rem : 0;
 }
 
+// How the tiled part of a batch of `count` base products with output extent M is launched on a device
+// with `sms` SMs: all leaves on the 64 x 64 tiling (two CTAs per SM), or `wide_leaves` leaves on the
+// 128 x 128 tiling followed by the rest on the 64 x 64 tiling.
+struct GemmSplit {
+    bool all_small;
+    int64_t wide_leaves;
+};
+inline GemmSplit gemm_split(int64_t M, int64_t count, int sms)
+{
+    // Few large tiles leave SMs idle: when the 128 x 128 tiling cannot give every SM a tile, the 64 x 64
+    // tiling is compared by rounds x tile cost (a 128 x 128 tile alone on an SM = 8 units).
+    const int64_t tpl_wide = ((M + 127) / 128) * ((M + 127) / 128), tpl_small = ((M + 63) / 64) * ((M + 63) / 64);
+    const int64_t t_wide = tpl_wide * count, t_small = tpl_small * count;
+    const int64_t cost_wide = ((t_wide + sms - 1) / sms) * 8;
+    const int64_t cost_small = t_small <= sms ? 2 : ((t_small + 2 * sms - 1) / (2 * sms)) * 4 + 1;
+    if (cost_small * 10 < cost_wide * 9) return GemmSplit{true, 0};
+    // The last, partly filled round of 128 x 128 tiles costs a whole tile time.  When it is less than half
+    // full, the leaves it belongs to go to the 64 x 64 tiling instead: full rounds of large tiles first, then
+    // a short launch of quarter-size tiles spread over all SMs.
+    const int64_t full_rounds = t_wide / sms, left = t_wide - full_rounds * sms;
+    int64_t wide_leaves = count;
+    if (full_rounds >= 4 && left > 0 && 2 * left < sms) {
+        wide_leaves = full_rounds * sms / tpl_wide;
+        if ((count - wide_leaves) * tpl_small > 2 * int64_t(sms)) wide_leaves = count;   // tail too long to pay off
+    }
+    return GemmSplit{false, wide_leaves};
+}
+constexpr int kNominalSMs = 148;   // B200; used where launches are counted without a device at hand
+
 // Kernels one replay of `op` launches (host arithmetic only; mirrors the launchers).
 int launches_of(const Launch &op);
 

@@ -30,6 +30,19 @@ def test_base_product_sizes(n, dist):
     check_full(n, max(n, 1), "", dist, 100 + n)
 
 
+@pytest.mark.parametrize("n", [65, 72, 136, 194, 260, 388, 771])
+def test_base_product_thin_remainders(n):
+    """Sizes 1..8 past a multiple of 64: tiled bulk plus thin products for the last rows / columns."""
+    check_full(n, n, "", "int8", 300 + n)
+    check_full(n, n, "", "normal", 301 + n, batch=3)
+
+
+def test_base_product_split_between_tile_shapes():
+    # 5 x 30 x 30... enough 128-tiles for >= 4 full rounds of 148 plus a short tail that moves to 64 x 64 tiles
+    check_full(512, 512, "", "int8", 77, batch=38)       # 608 tiles = 4 rounds + 16
+    check_full(256, 256, "", "uniform", 78, batch=150)   # 600 tiles = 4 rounds + 8
+
+
 def test_base_product_batch_spans_many_tiles():
     check_full(200, 256, "", "int8", 7, batch=40)
     check_full(384, 512, "", "uniform", 8, batch=9)

@@ -129,12 +129,13 @@ def test_launch_lists():
     # all BFS, one pass per level: one form and one recombine per level, one batched product launch
     single = binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES
     p = Plan(4096, 512, "BBB", flags=single)
-    assert p.launches_by_kind() == {"form": 3, "gemm": 1, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0}
-    assert p.launch_count == 7
+    # (343 x 16 tiles = 37 full rounds of 148 + 12: the leaf owning the leftover runs as a second, small-tile launch)
+    assert p.launches_by_kind() == {"form": 3, "gemm": 2, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0}
+    assert p.launch_count == 8
     p.close()
     # default: the two deepest BFS levels share one formation pass and one recombination pass
     p = Plan(4096, 512, "BBB")
-    assert p.launches_by_kind() == {"form": 2, "gemm": 1, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0}
+    assert p.launches_by_kind() == {"form": 2, "gemm": 2, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0}
     p.close()
     # DFS on top: 7 x (form_one [not for j = 0, 1], sub-tree, accumulate)
     p = Plan(16384, 512, "DBBBB", flags=single)
