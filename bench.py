@@ -183,6 +183,7 @@ def main():
     ap.add_argument("--no-cublas", action="store_true", help="skip the cuBLAS DGEMM comparator")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-probes", action="store_true", help="skip the FP64 rate probes")
+    ap.add_argument("--no-autotune", action="store_true", help="skip the measured choice of steps and interleaving")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -301,6 +302,22 @@ def main():
                   "max_abs_diff_vs_ours": float((Cc - C).abs().max()) if n <= 16384 else None}
         del Cc
 
+    tuned = None
+    if not args.no_autotune and batch * n * n * 8 * 3 < 20e9:
+        # the paper tunes every point to the best interleaving and number of Strassen steps (Section 5.4);
+        # reported beside the prescribed configuration, never instead of it
+        try:
+            ws_budget = max(plan.workspace_bytes, int(min(40e9, torch.cuda.mem_get_info()[0] - 2e9)))
+            ws = torch.empty(ws_budget, dtype=torch.uint8, device=dev)
+            Ct = torch.empty_like(A)
+            best, log = binding.strassen_autotune(n, A.data_ptr(), B.data_ptr(), Ct.data_ptr(), ws.data_ptr(), ws_budget,
+                                                  stream.cuda_stream, batch, 256, 3, 60.0)
+            tuned = dict(best, candidates=len(log), gflops=2.0 * n ** 3 * batch / (best["ms"] * 1e-3) / 1e9,
+                         workspace_budget_bytes=ws_budget)
+            del ws, Ct
+        except Exception as exc:
+            tuned = {"error": str(exc)}
+
     cpu = None
     if not args.no_cpu_baseline:
         import oracle
@@ -337,6 +354,7 @@ def main():
                           "hbm_gbs": hbm_gbs, "hbm_source": hbm_src,
                           "kernel_ms_per_step": {k: v / args.steps for k, v in kinds.items()}},
         "actual_gflops": (f_base + 15 * b_alg / (27 * 8)) / (ms * 1e-3) / 1e9 * world,
+        "autotuned": tuned,
         "cublas_dgemm": cublas,
         "vs_cublas": (cublas["ms"] / ms_local) if cublas else None,
         "cpu_baseline": cpu,

@@ -176,6 +176,41 @@ int strassen_plan_set_timing(strassen_plan *plan, int enabled);
 int strassen_plan_get_timings(strassen_plan *plan, double *ms_out /* [STRASSEN_K_COUNT] */);
 
 /*
+ * strassen_autotune -- choose the number of Strassen steps and the BFS/DFS interleaving by
+ * measurement [Section 5.4: "tuned to use the best interleaving pattern of BFS and DFS steps, and
+ * the best total number of Strassen steps"; Section 3.1 on interleaving].
+ *
+ * Candidates: for every step count L whose base size floor(n / 2^L) is >= min_base, every string of
+ * L characters over {B, D} whose workspace fits `workspace_bytes`.  Each candidate runs once to warm
+ * up and `repetitions` more times on `stream`, timed with CUDA events; the fastest run counts.  The
+ * search stops early after `max_seconds`.  On return *best holds the winner, `log` (if given) the
+ * first log_capacity candidates in search order, and C the product computed with the winner's plan
+ * (the stream is synchronised).  A, B, C: device pointers as for strassen_dgemm with ld = n; the
+ * caller owns them and the workspace.  Synchronous; allocates only the per-plan node tables.
+ */
+typedef struct strassen_tune_request {
+    int64_t n, batch;          /* batch 0 means 1                                            */
+    int64_t min_base;          /* smallest base size considered; 0 means 128                 */
+    int repetitions;           /* timed runs per candidate; 0 means 2                        */
+    double max_seconds;        /* 0 means 60                                                 */
+    const double *A, *B;
+    double *C;
+    void *workspace;           /* device memory, 256-byte aligned (may be NULL if bytes == 0) */
+    size_t workspace_bytes;
+    void *stream;
+} strassen_tune_request;
+
+typedef struct strassen_tune_entry {
+    int64_t cutoff;            /* pass to strassen_plan_create together with schedule        */
+    int levels;
+    char schedule[36];
+    double ms;                 /* best measured time of one product                          */
+} strassen_tune_entry;
+
+int strassen_autotune(const strassen_tune_request *request, strassen_tune_entry *best, strassen_tune_entry *log,
+                      int log_capacity, int *log_count);
+
+/*
  * strassen_probe_fp64 -- measure the FP64 arithmetic rate of the current device with a
  * register-resident loop (no memory traffic): kind 0 = scalar fused multiply-add, kind 1..4 =
  * the FP64 tensor-core instruction mma.sync m8n8k4 / m16n8k4 / m16n8k8 / m16n8k16.  Runs

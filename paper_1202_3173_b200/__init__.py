@@ -10,7 +10,7 @@ from __future__ import annotations
 from . import binding
 from .binding import StrassenError  # noqa: F401
 
-__all__ = ["Plan", "matmul", "binding", "StrassenError"]
+__all__ = ["Plan", "matmul", "autotune", "binding", "StrassenError"]
 
 
 class Plan:
@@ -125,3 +125,20 @@ def matmul(A, B, cutoff=512, schedule=None, workspace_budget_bytes=0):
     finally:
         plan.close()
     return C
+
+
+def autotune(A, B, workspace_budget_bytes, min_base=0, repetitions=0, max_seconds=0.0):
+    """Measure every (number of Strassen steps, BFS/DFS string) candidate that fits the budget on
+    A @ B and return (best, log, C): dicts with cutoff / levels / schedule / ms, and the product
+    computed with the winning plan.  torch supplies C and the workspace; the search itself runs
+    inside the library (strassen_autotune)."""
+    import torch
+    batch = 1 if A.dim() == 2 else A.shape[0]
+    n = A.shape[-1]
+    C = torch.empty_like(A)
+    ws = torch.empty(max(int(workspace_budget_bytes), 256), dtype=torch.uint8, device=A.device)
+    with torch.cuda.device(A.device):
+        stream = torch.cuda.current_stream().cuda_stream
+        best, log = binding.strassen_autotune(n, A.data_ptr(), B.data_ptr(), C.data_ptr(), ws.data_ptr(),
+                                              int(workspace_budget_bytes), stream, batch, min_base, repetitions, max_seconds)
+    return best, log, C

@@ -31,6 +31,18 @@ class strassen_options(ctypes.Structure):
                 ("workspace_budget_bytes", _sz), ("flags", _i64)]
 
 
+class strassen_tune_request(ctypes.Structure):
+    _fields_ = [("n", _i64), ("batch", _i64), ("min_base", _i64), ("repetitions", _int), ("max_seconds", ctypes.c_double),
+                ("A", _vp), ("B", _vp), ("C", _vp), ("workspace", _vp), ("workspace_bytes", _sz), ("stream", _vp)]
+
+
+class strassen_tune_entry(ctypes.Structure):
+    _fields_ = [("cutoff", _i64), ("levels", _int), ("schedule", ctypes.c_char * 36), ("ms", ctypes.c_double)]
+
+    def as_dict(self):
+        return {"cutoff": int(self.cutoff), "levels": int(self.levels), "schedule": self.schedule.decode(), "ms": float(self.ms)}
+
+
 SYMBOLS = [
     ("strassen_plan_create", _vp, [_i64, _i64, _cp]),
     ("strassen_plan_create_ex", _vp, [ctypes.POINTER(strassen_options)]),
@@ -49,6 +61,8 @@ SYMBOLS = [
     ("strassen_schedule_model_bytes", _sz, [_i64, _i64, _i64, _cp, _int]),
     ("strassen_plan_set_timing", _int, [_vp, _int]),
     ("strassen_plan_get_timings", _int, [_vp, _dp]),
+    ("strassen_autotune", _int, [ctypes.POINTER(strassen_tune_request), ctypes.POINTER(strassen_tune_entry),
+                                 ctypes.POINTER(strassen_tune_entry), _int, ctypes.POINTER(_int)]),
     ("strassen_probe_fp64", _int, [_int, _i64, _vp, _dp]),
     ("strassen_dgemm_static", _int, [_i64, _vp, _vp, _vp, _vp]),
     ("strassen_last_error", _cp, []),
@@ -180,6 +194,17 @@ def strassen_dgemm_static(n: int, A: int, B: int, C: int, stream: int = 0) -> No
     """One Strassen-Winograd level with all temporaries in the library's static device array:
     for callers that must not allocate device memory.  A, B, C: device addresses, rows of n."""
     _check(lib().strassen_dgemm_static(n, A, B, C, stream))
+
+
+def strassen_autotune(n, A, B, C, workspace, workspace_bytes, stream=0, batch=1, min_base=0, repetitions=0,
+                      max_seconds=0.0, log_capacity=256):
+    """Returns (best, log): dicts with cutoff / levels / schedule / ms.  A, B, C, workspace: device addresses."""
+    req = strassen_tune_request(n, batch, min_base, repetitions, max_seconds, A, B, C, workspace, workspace_bytes, stream)
+    best = strassen_tune_entry()
+    log = (strassen_tune_entry * max(log_capacity, 1))()
+    count = _int(0)
+    _check(lib().strassen_autotune(ctypes.byref(req), ctypes.byref(best), log, log_capacity, ctypes.byref(count)))
+    return best.as_dict(), [log[i].as_dict() for i in range(count.value)]
 
 
 def strassen_probe_fp64(kind: int, iters: int, stream: int = 0) -> float:

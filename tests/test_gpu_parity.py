@@ -186,6 +186,26 @@ def test_timing_split_sums_to_about_the_total():
     assert t["gemm"] > 0 and t["form"] > 0 and t["recombine"] > 0 and t["peel"] == 0
 
 
+def test_autotune_returns_a_valid_fastest_candidate():
+    from paper_1202_3173_b200 import autotune
+    n = 1024
+    A, B = inputs.pair(n, "uniform", 91, device="cuda")
+    best, log, C = autotune(A, B, workspace_budget_bytes=int(1e9), min_base=128, repetitions=2)
+    assert len(log) == 1 + 2 + 4 + 8                       # L = 0..3, every B/D string
+    assert {e["levels"] for e in log} == {0, 1, 2, 3}
+    assert best["ms"] == min(e["ms"] for e in log) and best["ms"] > 0
+    assert len(best["schedule"]) == best["levels"] and set(best["schedule"]) <= set("BD")
+    # the tuned pair recreates a plan, and C holds that plan's (correct) product
+    plan = Plan(n, best["cutoff"], best["schedule"])
+    assert plan.levels == best["levels"]
+    plan.close()
+    ref = oracle.classical(A.cpu().numpy(), B.cpu().numpy())
+    assert float(np.abs(C.cpu().numpy() - ref).max()) <= bound(n, A, B)
+    # a budget too small for any recursion leaves only the classical product
+    best0, log0, _ = autotune(A, B, workspace_budget_bytes=0, min_base=128)
+    assert best0["levels"] == 0 and len(log0) == 1
+
+
 # ---- full-size configurations: sampled blocks of the definition + exact integer variant ----
 
 def test_config_n4096_bbb_full_size():

@@ -47,6 +47,16 @@ def test_null_arguments_are_reported_not_crashed():
     assert l.strassen_plan_workspace_bytes(None) == 0
 
 
+def test_autotune_rejects_bad_requests_without_a_device():
+    l = binding.lib()
+    assert l.strassen_autotune(None, None, None, 0, None) == -1
+    req = binding.strassen_tune_request(64, 1, 0, 0, 0.0, None, None, None, None, 0, None)
+    best = binding.strassen_tune_entry()
+    import ctypes
+    assert l.strassen_autotune(ctypes.byref(req), ctypes.byref(best), None, 0, None) == -1
+    assert b"non-NULL" in l.strassen_last_error()
+
+
 def test_alias_and_alignment_checks_come_before_any_device_work():
     p = Plan(64, 16, "BB")
     l = binding.lib()
