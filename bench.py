@@ -240,23 +240,35 @@ def main():
     plan.set_timing(False)
     ms = reduce_max(ms_local, dev)
 
-    # ---- end to end: host buffers, copies inside the timed region ----------------------------
-    e2e_ms = None
-    if not args.no_e2e:
+    hA = hB = None
+    if not args.no_e2e or (rank == 0 and not args.no_cpu_baseline):
         hA, hB = A.cpu().pin_memory(), B.cpu().pin_memory()
-        hC = torch.empty_like(hA).pin_memory()
-        e2e_steps = max(3, min(args.steps, 10))
-        for _ in range(2):
-            plan.run_host(hA, hB, hC)
-        barrier()
-        ev0.record(stream)
-        for _ in range(e2e_steps):
-            plan.run_host(hA, hB, hC)
-        ev1.record(stream)
-        barrier()
-        e2e_ms = reduce_max(ev0.elapsed_time(ev1) / e2e_steps, dev)
+
+    def run_e2e():
+        """Host buffers, copies inside the timed region.  Runs last: the device copies of A, B, C are freed
+        first so that the library's staging buffers fit beside the workspace at the largest size."""
+        nonlocal A, B, C
+        if args.no_e2e:
+            return None, None
+        try:
+            del A, B, C
+            torch.cuda.empty_cache()
+            hC = torch.empty_like(hA).pin_memory()
+            e2e_steps = max(3, min(args.steps, 10))
+            for _ in range(2):
+                plan.run_host(hA, hB, hC)
+            barrier()
+            ev0.record(stream)
+            for _ in range(e2e_steps):
+                plan.run_host(hA, hB, hC)
+            ev1.record(stream)
+            barrier()
+            return reduce_max(ev0.elapsed_time(ev1) / e2e_steps, dev), None
+        except Exception as exc:           # out of device or pinned memory at the largest sizes
+            return None, str(exc)
 
     if rank != 0:
+        run_e2e()
         plan.close()
         if world > 1:
             dist.destroy_process_group()
@@ -321,29 +333,33 @@ def main():
     cpu = None
     if not args.no_cpu_baseline:
         import oracle
-        a_h = (A if batch == 1 else A[0]).cpu().numpy()
-        b_h = (B if batch == 1 else B[0]).cpu().numpy()
+        a_h = (hA if batch == 1 else hA[0]).numpy()
+        b_h = (hB if batch == 1 else hB[0]).numpy()
         g, rows, secs = time_oracle_slab(n, a_h, b_h)
         cpu = {"value": g, "unit": UNIT, "cores": oracle.cores(), "kind": "oracle",
                "sample": "classical oracle on the first %d of %d rows of one product (%.1f s); classical flops "
                          "equal effective flops, so the rate stands for the whole product" % (rows, n, secs)}
 
+    launches_by_kind, launch_count, sched_resolved, level_list, ws_bytes = (plan.launches_by_kind(), plan.launch_count,
+                                                                       plan.schedule, plan.level_sizes, plan.workspace_bytes)
+    e2e_ms, e2e_error = run_e2e()
     ours_gflops = whole_job_value(n, batch, ms, world)
     line = {
         "metric": METRIC, "value": ours_gflops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": describe(args.workload), "schedule": plan.schedule, "levels": plan.level_sizes,
-                   "workspace_bytes": plan.workspace_bytes,
+        "config": {"workload": describe(args.workload), "schedule": sched_resolved, "levels": level_list,
+                   "workspace_bytes": ws_bytes,
                    "l2": "inputs larger than L2 (A+B+C %.0f MB + workspace)" % (3 * batch * n * n * 8 / 1e6)
                          if 3 * batch * n * n * 8 > 126e6 else "L2-resident problem (A+B+C %.1f MB): launch-bound"
                          % (3 * batch * n * n * 8 / 1e6),
                    "parallelism": "replicas only (no collective)" if world > 1 else "single GPU"},
         "clocks": clocks,
+        "e2e_error": e2e_error,
         "e2e": None if e2e_ms is None else
                {"value": whole_job_value(n, batch, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 2 * batch * n * n * 8, "d2h_bytes_per_step": batch * n * n * 8},
-        "gpu_launches": args.steps * plan.launch_count,
+        "gpu_launches": args.steps * launch_count,
         "roofline": {"bound": "alu", "kernel": "gemm_f64_kernel (batched base products)", "achieved": achieved_tflops,
                      "peak": FP64_PEAK_NOMINAL_TFLOPS, "unit": "TFLOP/s", "frac": achieved_tflops / FP64_PEAK_NOMINAL_TFLOPS,
                      "peak_source": "148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz (unit counts and max clock)",
