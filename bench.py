@@ -184,6 +184,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-probes", action="store_true", help="skip the FP64 rate probes")
     ap.add_argument("--no-autotune", action="store_true", help="skip the measured choice of steps and interleaving")
+    ap.add_argument("--graph", action="store_true", help="also time the plan replayed as one CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -330,6 +331,22 @@ def main():
         except Exception as exc:
             tuned = {"error": str(exc)}
 
+    graph_ms = None
+    if args.graph:
+        gplan = Plan(n, cutoff, plan.schedule, batch=batch, flags=binding.STRASSEN_FLAG_CUDA_GRAPH)
+        Cg = torch.empty_like(A)
+        for _ in range(3):
+            gplan(A, B, out=Cg)
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            gplan(A, B, out=Cg)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        graph_ms = ev0.elapsed_time(ev1) / args.steps
+        gplan.close()
+        del Cg
+
     cpu = None
     if not args.no_cpu_baseline:
         import oracle
@@ -371,6 +388,7 @@ def main():
                           "kernel_ms_per_step": {k: v / args.steps for k, v in kinds.items()}},
         "actual_gflops": (f_base + 15 * b_alg / (27 * 8)) / (ms * 1e-3) / 1e9 * world,
         "autotuned": tuned,
+        "cuda_graph_ms_per_step": graph_ms,
         "cublas_dgemm": cublas,
         "vs_cublas": (cublas["ms"] / ms_local) if cublas else None,
         "cpu_baseline": cpu,

@@ -83,6 +83,14 @@ typedef struct strassen_options {
  * the same order, bit-identical results).  This flag keeps one pass per level. */
 #define STRASSEN_FLAG_SINGLE_LEVEL_PASSES 1
 
+/* Replay the plan's launch list as one CUDA graph: the first strassen_dgemm call with a given
+ * (A, B, C, workspace) captures the launches on an internal stream and instantiates the graph; that
+ * call and every later one with the same pointers costs a single graph launch on the caller's
+ * stream (different pointers re-capture).  Meant for launch-bound plans: small n, or DFS-heavy
+ * schedules with hundreds of launches.  Per-family timing is not available in this mode (a call
+ * made while timing is enabled is enqueued launch by launch). */
+#define STRASSEN_FLAG_CUDA_GRAPH 2
+
 /*
  * strassen_plan_create -- plan C = A.B for n x n matrices [Algorithm 1 "Require A, B n x n"].
  *   n        matrix size (>= 1), contiguous rows (ld = n), one product per call.

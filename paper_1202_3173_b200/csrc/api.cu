@@ -47,6 +47,10 @@ struct strassen_plan {
     bool timing = false;
     std::vector<TimedLaunch> pending;
     std::vector<cudaEvent_t> free_events;
+    bool use_graph = false;               // STRASSEN_FLAG_CUDA_GRAPH
+    cudaStream_t capture_stream = nullptr;
+    cudaGraphExec_t graph_exec = nullptr;
+    const void *graph_ptrs[4] = {nullptr, nullptr, nullptr, nullptr};   // A, B, C, workspace the graph was captured for
     double acc_ms[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0};
     int64_t launches[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0};
     int64_t launch_total = 0;
@@ -100,6 +104,8 @@ int ensure_device_state(strassen_plan *p)
             return fail(STRASSEN_CUDA_ERROR, "this library holds sm_100a code only; the current device is not a B200-class GPU");
         e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        e = configure_gemm_kernels();       // opt-in to large dynamic shared memory, outside any capture
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute");
         p->device = dev;
     }
     if (!p->d_tab) {
@@ -121,6 +127,76 @@ int ensure_device_state(strassen_plan *p)
         p->ws_bytes = need;
         p->own_ws = true;
     }
+    return STRASSEN_OK;
+}
+
+// Enqueue every launch of the plan on `stream` (optionally bracketed by timing events).
+int enqueue_launches(strassen_plan *p, const Bases &bases, bool bases16, cudaStream_t stream, bool timed)
+{
+    int launched = 0;
+    for (const Launch &op : p->d.launches) {
+        const bool vec = op.vec_ok && bases16;
+        TimedLaunch t{family(op.kind), nullptr, nullptr};
+        if (timed) {
+            t.start = take_event(p);
+            t.stop = take_event(p);
+            cudaEventRecord(t.start, stream);
+        }
+        cudaError_t e = cudaSuccess;
+        switch (op.kind) {
+        case OP_FORM: e = launch_form(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_GEMM: e = launch_gemm(p->d_tab, op, bases, p->sm_count, stream, &launched); break;
+        case OP_RECOMBINE: e = launch_recombine(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_FORM_ONE: e = launch_form_one(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_ACCUMULATE: e = launch_accumulate(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_PEEL: e = launch_peel(p->d_tab, op, bases, stream, &launched); break;
+        case OP_FORM2: e = launch_form2(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
+        }
+        if (timed) {
+            cudaEventRecord(t.stop, stream);
+            p->pending.push_back(t);
+        }
+        if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    }
+    return STRASSEN_OK;
+}
+
+// STRASSEN_FLAG_CUDA_GRAPH: the launch list is captured once per (A, B, C, workspace) into a CUDA graph on
+// an internal stream and replayed on the caller's stream with a single launch.
+int replay_graph(strassen_plan *p, const Bases &bases, bool bases16, cudaStream_t stream)
+{
+    bool same = p->graph_exec != nullptr;
+    for (int i = 0; i < 4; ++i) same = same && p->graph_ptrs[i] == bases.p[i];
+    if (!same) {
+        if (!p->capture_stream) {
+            cudaError_t e = cudaStreamCreateWithFlags(&p->capture_stream, cudaStreamNonBlocking);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaStreamCreate(capture)");
+        }
+        if (p->graph_exec) {
+            cudaGraphExecDestroy(p->graph_exec);
+            p->graph_exec = nullptr;
+        }
+        cudaError_t e = cudaStreamBeginCapture(p->capture_stream, cudaStreamCaptureModeThreadLocal);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaStreamBeginCapture");
+        const int rc = enqueue_launches(p, bases, bases16, p->capture_stream, false);
+        cudaGraph_t graph = nullptr;
+        e = cudaStreamEndCapture(p->capture_stream, &graph);
+        if (rc != STRASSEN_OK) {
+            if (graph) cudaGraphDestroy(graph);
+            return rc;
+        }
+        if (e != cudaSuccess || !graph) return cuda_fail(e, "cudaStreamEndCapture");
+        e = cudaGraphInstantiate(&p->graph_exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) {
+            p->graph_exec = nullptr;
+            return cuda_fail(e, "cudaGraphInstantiate");
+        }
+        for (int i = 0; i < 4; ++i) p->graph_ptrs[i] = bases.p[i];
+    }
+    cudaError_t e = cudaGraphLaunch(p->graph_exec, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGraphLaunch");
     return STRASSEN_OK;
 }
 
@@ -160,6 +236,7 @@ strassen_plan *create(const strassen_options &o)
         return nullptr;
     }
     d.fuse_two_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) == 0;
+    p->use_graph = (o.flags & STRASSEN_FLAG_CUDA_GRAPH) != 0;
     d.sizes = level_sizes(n, cutoff);
     const size_t L = d.sizes.size() - 1;
     const bool want_auto = !o.schedule || strcmp(o.schedule, "auto") == 0;
@@ -263,33 +340,8 @@ int strassen_dgemm(strassen_plan *p, const double *A, const double *B, double *C
     bases.p[BASE_C] = C;
     bases.p[BASE_WS] = p->ws;
     const bool bases16 = ((bits | reinterpret_cast<uintptr_t>(p->ws)) & 15) == 0;
-    int launched = 0;
-    for (const Launch &op : d.launches) {
-        const bool vec = op.vec_ok && bases16;
-        TimedLaunch t{family(op.kind), nullptr, nullptr};
-        if (p->timing) {
-            t.start = take_event(p);
-            t.stop = take_event(p);
-            cudaEventRecord(t.start, stream);
-        }
-        cudaError_t e = cudaSuccess;
-        switch (op.kind) {
-        case OP_FORM: e = launch_form(p->d_tab, op, bases, vec, stream, &launched); break;
-        case OP_GEMM: e = launch_gemm(p->d_tab, op, bases, p->sm_count, stream, &launched); break;
-        case OP_RECOMBINE: e = launch_recombine(p->d_tab, op, bases, vec, stream, &launched); break;
-        case OP_FORM_ONE: e = launch_form_one(p->d_tab, op, bases, vec, stream, &launched); break;
-        case OP_ACCUMULATE: e = launch_accumulate(p->d_tab, op, bases, vec, stream, &launched); break;
-        case OP_PEEL: e = launch_peel(p->d_tab, op, bases, stream, &launched); break;
-        case OP_FORM2: e = launch_form2(p->d_tab, op, bases, vec, stream, &launched); break;
-        case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
-        }
-        if (p->timing) {
-            cudaEventRecord(t.stop, stream);
-            p->pending.push_back(t);
-        }
-        if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
-    }
-    return STRASSEN_OK;
+    if (p->use_graph && !p->timing) return replay_graph(p, bases, bases16, stream);
+    return enqueue_launches(p, bases, bases16, stream, p->timing);
 }
 
 int strassen_dgemm_host(strassen_plan *p, const double *hA, const double *hB, double *hC, void *stream_v)
@@ -347,6 +399,8 @@ void strassen_plan_destroy(strassen_plan *p)
         cudaEventDestroy(t.stop);
     }
     for (cudaEvent_t e : p->free_events) cudaEventDestroy(e);
+    if (p->graph_exec) cudaGraphExecDestroy(p->graph_exec);
+    if (p->capture_stream) cudaStreamDestroy(p->capture_stream);
     if (p->d_tab) cudaFree(p->d_tab);
     if (p->own_ws && p->ws) cudaFree(p->ws);
     if (p->stage_a) cudaFree(p->stage_a);
@@ -373,7 +427,7 @@ int strassen_plan_set_workspace(strassen_plan *p, void *device_ptr, size_t bytes
     if (p->own_ws && p->ws) cudaFree(p->ws);
     p->ws = static_cast<double *>(device_ptr);
     p->ws_bytes = bytes;
-    p->own_ws = false;
+    p->own_ws = false;       // a captured graph is re-captured on the next call (its workspace pointer differs)
     return STRASSEN_OK;
 }
 

@@ -313,18 +313,24 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
 
 namespace {
 
+bool g_configured[64];   // per device: kernels opted in to > 48 KB of dynamic shared memory
+
+}  // namespace
+
+cudaError_t configure_gemm_kernels();
+
+namespace {
+
 template <class C>
 cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, int K, long long count, int sm_count,
                        cudaStream_t stream)
 {
-    static bool configured[64] = {false};   // per device: opt in to > 48 KB of dynamic shared memory
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(gemm_f64_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::SMEM_BYTES));
+    if (dev < 0 || dev >= 64 || !g_configured[dev]) {
+        e = configure_gemm_kernels();
         if (e != cudaSuccess) return e;
-        if (dev < 64) configured[dev] = true;
     }
     const int tiles_m = (M + C::BM - 1) / C::BM, tiles_n = (M + C::BN - 1) / C::BN;
     const int tiles_per_node = tiles_m * tiles_n;
@@ -337,6 +343,20 @@ cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, int K, long
 }
 
 }  // namespace
+
+cudaError_t configure_gemm_kernels()
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && g_configured[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(gemm_f64_kernel<CfgWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgWide::SMEM_BYTES));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemm_f64_kernel<CfgSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgSmall::SMEM_BYTES));
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) g_configured[dev] = true;
+    return cudaSuccess;
+}
 
 cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
                         int *launched)

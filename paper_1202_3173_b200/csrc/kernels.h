@@ -78,6 +78,9 @@ inline GemmSplit gemm_split(int64_t M, int64_t count, int sms)
 }
 constexpr int kNominalSMs = 148;   // B200; used where launches are counted without a device at hand
 
+// Sets the shared-memory attribute of every GEMM kernel shape on the current device (idempotent).
+cudaError_t configure_gemm_kernels();
+
 // Kernels one replay of `op` launches (host arithmetic only; mirrors the launchers).
 int launches_of(const Launch &op);
 

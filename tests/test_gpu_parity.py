@@ -142,6 +142,30 @@ def test_batch_with_two_level_passes():
     check_full(260, 65, "BB", "int8", 122, batch=3)      # odd quarter size: 8-byte accesses
 
 
+def test_cuda_graph_replay_matches_launch_by_launch():
+    n = 512
+    A, B = inputs.pair(n, "uniform", 131, device="cuda")
+    A2, B2 = inputs.pair(n, "int8", 133, device="cuda")
+    for cutoff, sched in ((256, "B"), (64, "DBD"), (32, "DDDD")):
+        eager = Plan(n, cutoff, sched)
+        graph = Plan(n, cutoff, sched, flags=binding.STRASSEN_FLAG_CUDA_GRAPH)
+        want = eager(A, B).clone()
+        C = torch.empty_like(A)
+        for _ in range(3):                       # capture on the first call, replay afterwards
+            C.fill_(float("nan"))
+            graph(A, B, out=C)
+            torch.cuda.synchronize()
+            assert torch.equal(C, want)
+        # other pointers: the graph is captured again and stays correct
+        C2 = graph(A2, B2)
+        torch.cuda.synchronize()
+        assert np.array_equal(C2.cpu().numpy(), oracle.classical(A2.cpu().numpy(), B2.cpu().numpy()))
+        graph(A, B, out=C)
+        torch.cuda.synchronize()
+        assert torch.equal(C, want)
+        eager.close(); graph.close()
+
+
 def test_schedules_agree_exactly_on_integers():
     A, B = inputs.pair(512, "int8", 41, device="cuda")
     outs = [run_plan(512, 64, s, A, B) for s in ("BBB", "DDD", "BDB", "DBD")]
