@@ -443,15 +443,20 @@ __global__ void __launch_bounds__(256) thin_cols_kernel(const Node *__restrict__
             bs[t][k] = t < nc ? B[int64_t(k0 + k) * nd.b.ld + c0 + t] : 0.0;
         }
         __syncthreads();
+        // k outer, the warp's 4 rows inner: the staged B values are read from shared memory once per k
+        const double *a0 = A + int64_t(min(rbase, rows - 1)) * nd.a.ld + k0;
+        const int64_t lda = nd.a.ld;
+        const int nrow = min(4, rows - rbase);
+        for (int k = lane; k < kn; k += 32) {
+            double bv[NC];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int r = rbase + i;
-            if (r < rows) {
-                const double *a = A + int64_t(r) * nd.a.ld + k0;
-                for (int k = lane; k < kn; k += 32) {
-                    const double av = a[k];
+            for (int t = 0; t < NC; ++t) bv[t] = bs[t][k];
 #pragma unroll
-                    for (int t = 0; t < NC; ++t) acc[i][t] = fma(av, bs[t][k], acc[i][t]);
+            for (int i = 0; i < 4; ++i) {
+                if (i < nrow) {
+                    const double av = a0[int64_t(i) * lda + k];
+#pragma unroll
+                    for (int t = 0; t < NC; ++t) acc[i][t] = fma(av, bv[t], acc[i][t]);
                 }
             }
         }
@@ -469,53 +474,77 @@ __global__ void __launch_bounds__(256) thin_cols_kernel(const Node *__restrict__
     }
 }
 
-// Rows [r0, r0 + nr) of C for columns [0, cols): a thread owns one column and every TR_SLICES-th k;
-// the slices are summed through shared memory in a fixed order.
-constexpr int TR_COLS = 32, TR_SLICES = 16;
+// Rows [r0, r0 + nr) of C for columns [0, cols): a thread owns two adjacent columns and one of
+// TR_SLICES interleaved pairs of k; the nr rows of A are staged through shared memory in chunks (read
+// back as broadcast 16-byte pairs), and the slices are summed through shared memory in a fixed order.
+constexpr int TR_COLS = 64, TR_SLICES = 8, TR_CHUNK = 512;
 template <int NR>
-__global__ void __launch_bounds__(TR_COLS *TR_SLICES) thin_rows_kernel(const Node *__restrict__ nodes, Bases bases, int K,
-                                                                      int cols, int r0, int nr, int item0)
+__global__ void __launch_bounds__((TR_COLS / 2) * TR_SLICES) thin_rows_kernel(const Node *__restrict__ nodes, Bases bases,
+                                                                              int K, int cols, int r0, int nr, int item0)
 {
-    __shared__ double part[TR_SLICES][NR][TR_COLS + 1];
+    // one buffer, used first for the staged rows of A and, after the k loop, for the slice sums
+    constexpr int AS_WORDS = NR * TR_CHUNK, PART_WORDS = TR_SLICES * NR * (TR_COLS + 2);
+    __shared__ __align__(16) double buf[AS_WORDS > PART_WORDS ? AS_WORDS : PART_WORDS];
+    double(*as)[TR_CHUNK] = reinterpret_cast<double(*)[TR_CHUNK]>(buf);
+    double(*part)[NR][TR_COLS + 2] = reinterpret_cast<double(*)[NR][TR_COLS + 2]>(buf);
     const Node nd = nodes[item0 + blockIdx.y];
     const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
     double *C = resolve(bases, nd.c);
-    const int c = blockIdx.x * TR_COLS + threadIdx.x;
-    double acc[NR];
+    const int tid = threadIdx.y * (TR_COLS / 2) + threadIdx.x;
+    const int c = blockIdx.x * TR_COLS + 2 * threadIdx.x;
+    const bool c0ok = c < cols, c1ok = c + 1 < cols;
+    const int64_t ldb = nd.b.ld, lda = nd.a.ld;
+    const double *b = B + (c0ok ? c : 0);
+    const int c1 = c1ok ? 1 : 0;
+    double acc[NR][2];
 #pragma unroll
-    for (int t = 0; t < NR; ++t) acc[t] = 0.0;
-    if (c < cols) {
-        const double *b = B + c;
-        const int64_t ldb = nd.b.ld, lda = nd.a.ld;
-        const double *arow = A + int64_t(r0) * lda;
-        int k = threadIdx.y;
-        for (; k + 3 * TR_SLICES < K; k += 4 * TR_SLICES) {
-            double bv[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) bv[u] = b[int64_t(k + u * TR_SLICES) * ldb];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int t = 0; t < NR; ++t)
-                    if (t < nr) acc[t] = fma(arow[int64_t(t) * lda + k + u * TR_SLICES], bv[u], acc[t]);
+    for (int t = 0; t < NR; ++t) acc[t][0] = acc[t][1] = 0.0;
+    for (int k0 = 0; k0 < K; k0 += TR_CHUNK) {
+        const int kn = min(TR_CHUNK, K - k0);
+        __syncthreads();
+        for (int e = tid; e < NR * TR_CHUNK; e += (TR_COLS / 2) * TR_SLICES) {
+            const int t = e / TR_CHUNK, k = e % TR_CHUNK;
+            as[t][k] = (t < nr && k < kn) ? A[int64_t(r0 + t) * lda + k0 + k] : 0.0;
         }
-        for (; k < K; k += TR_SLICES) {
-            const double bv = b[int64_t(k) * ldb];
+        __syncthreads();
+        if (c0ok) {
+            // slice s owns k = 2 s, 2 s + 1, then + 2 TR_SLICES, ...; entries past kn are zero in `as`
+            for (int k = 2 * threadIdx.y; k < kn; k += 2 * TR_SLICES) {
+                const double *bk = b + int64_t(k0 + k) * ldb;
+                const bool k1ok = k + 1 < kn;
+                const double b00 = bk[0], b01 = bk[c1];
+                const double b10 = k1ok ? bk[ldb] : 0.0, b11 = k1ok ? bk[ldb + c1] : 0.0;
 #pragma unroll
-            for (int t = 0; t < NR; ++t)
-                if (t < nr) acc[t] = fma(arow[int64_t(t) * lda + k], bv, acc[t]);
+                for (int t = 0; t < NR; ++t) {
+                    const double2 a2 = *reinterpret_cast<const double2 *>(&as[t][k]);
+                    acc[t][0] = fma(a2.x, b00, acc[t][0]);
+                    acc[t][1] = fma(a2.x, b01, acc[t][1]);
+                    acc[t][0] = fma(a2.y, b10, acc[t][0]);
+                    acc[t][1] = fma(a2.y, b11, acc[t][1]);
+                }
+            }
         }
     }
+    __syncthreads();    // everyone is done reading the staged rows
 #pragma unroll
-    for (int t = 0; t < NR; ++t) part[threadIdx.y][t][threadIdx.x] = acc[t];
+    for (int t = 0; t < NR; ++t) {
+        part[threadIdx.y][t][2 * threadIdx.x] = acc[t][0];
+        part[threadIdx.y][t][2 * threadIdx.x + 1] = acc[t][1];
+    }
     __syncthreads();
-    if (threadIdx.y == 0 && c < cols) {
+    if (threadIdx.y == 0 && c0ok) {
 #pragma unroll
         for (int t = 0; t < NR; ++t) {
-            double v = 0.0;
+            double v0 = 0.0, v1 = 0.0;
 #pragma unroll
-            for (int i = 0; i < TR_SLICES; ++i) v += part[i][t][threadIdx.x];
-            if (t < nr) C[int64_t(r0 + t) * nd.c.ld + c] = v;
+            for (int i = 0; i < TR_SLICES; ++i) {
+                v0 += part[i][t][2 * threadIdx.x];
+                v1 += part[i][t][2 * threadIdx.x + 1];
+            }
+            if (t < nr) {
+                C[int64_t(r0 + t) * nd.c.ld + c] = v0;
+                if (c1ok) C[int64_t(r0 + t) * nd.c.ld + c + 1] = v1;
+            }
         }
     }
 }
@@ -678,7 +707,7 @@ cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int c
 {
     const int64_t total = count;
     FOR_CHUNKS(total) {
-        const dim3 grid((cols + TR_COLS - 1) / TR_COLS, unsigned(zn)), block(TR_COLS, TR_SLICES);
+        const dim3 grid((cols + TR_COLS - 1) / TR_COLS, unsigned(zn)), block(TR_COLS / 2, TR_SLICES);
         if (nr <= 1) thin_rows_kernel<1><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
         else if (nr <= 2) thin_rows_kernel<2><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
         else if (nr <= 4) thin_rows_kernel<4><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
