@@ -241,6 +241,7 @@ def main():
     plan.set_timing(False)
     ms = reduce_max(ms_local, dev)
 
+    sched_resolved = plan.schedule
     hA = hB = None
     if not args.no_e2e or (rank == 0 and not args.no_cpu_baseline):
         hA, hB = A.cpu().pin_memory(), B.cpu().pin_memory()
@@ -250,23 +251,32 @@ def main():
         first so that the library's staging buffers fit beside the workspace at the largest size."""
         nonlocal A, B, C
         if args.no_e2e:
-            return None, None
+            return [None, None], None
         try:
             del A, B, C
             torch.cuda.empty_cache()
             hC = torch.empty_like(hA).pin_memory()
             e2e_steps = max(3, min(args.steps, 10))
-            for _ in range(2):
-                plan.run_host(hA, hB, hC)
-            barrier()
-            ev0.record(stream)
-            for _ in range(e2e_steps):
-                plan.run_host(hA, hB, hC)
-            ev1.record(stream)
-            barrier()
-            return reduce_max(ev0.elapsed_time(ev1) / e2e_steps, dev), None
+            out = []
+            for flags in (0, binding.STRASSEN_FLAG_HOST_PIPELINE):     # strictly in stream order, then pipelined
+                hplan = plan if flags == 0 else Plan(n, cutoff, sched_resolved, batch=batch, flags=flags)
+                if flags and 3 * batch * n * n * 8 * 2 > 60e9:
+                    out.append(None)                                  # two sets of device copies would not fit
+                    continue
+                for _ in range(2):
+                    hplan.run_host(hA, hB, hC)
+                barrier()
+                ev0.record(stream)
+                for _ in range(e2e_steps):
+                    hplan.run_host(hA, hB, hC)
+                ev1.record(stream)
+                barrier()
+                out.append(reduce_max(ev0.elapsed_time(ev1) / e2e_steps, dev))
+                if flags:
+                    hplan.close()
+            return out, None
         except Exception as exc:           # out of device or pinned memory at the largest sizes
-            return None, str(exc)
+            return [None, None], str(exc)
 
     if rank != 0:
         run_e2e()
@@ -357,9 +367,9 @@ def main():
                "sample": "classical oracle on the first %d of %d rows of one product (%.1f s); classical flops "
                          "equal effective flops, so the rate stands for the whole product" % (rows, n, secs)}
 
-    launches_by_kind, launch_count, sched_resolved, level_list, ws_bytes = (plan.launches_by_kind(), plan.launch_count,
-                                                                       plan.schedule, plan.level_sizes, plan.workspace_bytes)
-    e2e_ms, e2e_error = run_e2e()
+    launches_by_kind, launch_count, level_list, ws_bytes = (plan.launches_by_kind(), plan.launch_count, plan.level_sizes,
+                                                        plan.workspace_bytes)
+    (e2e_ms, e2e_pipe_ms), e2e_error = run_e2e()
     ours_gflops = whole_job_value(n, batch, ms, world)
     line = {
         "metric": METRIC, "value": ours_gflops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -374,8 +384,12 @@ def main():
         "clocks": clocks,
         "e2e_error": e2e_error,
         "e2e": None if e2e_ms is None else
-               {"value": whole_job_value(n, batch, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": 2 * batch * n * n * 8, "d2h_bytes_per_step": batch * n * n * 8},
+               {"value": whole_job_value(n, batch, e2e_pipe_ms or e2e_ms, world), "unit": UNIT,
+                "ms_per_step": e2e_pipe_ms or e2e_ms,
+                "mode": "strassen_dgemm_host, consecutive calls pipelined over plan-owned streams (STRASSEN_FLAG_HOST_PIPELINE)"
+                        if e2e_pipe_ms else "strassen_dgemm_host, everything in stream order",
+                "h2d_bytes_per_step": 2 * batch * n * n * 8, "d2h_bytes_per_step": batch * n * n * 8,
+                "in_order_ms_per_step": e2e_ms, "pipelined_ms_per_step": e2e_pipe_ms},
         "gpu_launches": args.steps * launch_count,
         "roofline": {"bound": "alu", "kernel": "gemm_f64_kernel (batched base products)", "achieved": achieved_tflops,
                      "peak": FP64_PEAK_NOMINAL_TFLOPS, "unit": "TFLOP/s", "frac": achieved_tflops / FP64_PEAK_NOMINAL_TFLOPS,

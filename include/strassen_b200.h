@@ -91,6 +91,15 @@ typedef struct strassen_options {
  * made while timing is enabled is enqueued launch by launch). */
 #define STRASSEN_FLAG_CUDA_GRAPH 2
 
+/* strassen_dgemm_host only: run consecutive host-buffer products as a pipeline over three streams
+ * owned by the plan -- the copy-in of call k+1 beside the products of call k and the copy-out of call
+ * k-1 (two sets of device copies; one if the device has no room for two).  `stream` then only waits
+ * for this call's result copy: work enqueued on it earlier is NOT waited for, so hostA / hostB must
+ * hold their final contents when the call is made, and the host buffers of a call must stay untouched
+ * until `stream` (or the device) has been synchronised.  Without this flag everything is enqueued on
+ * `stream` in order. */
+#define STRASSEN_FLAG_HOST_PIPELINE 4
+
 /*
  * strassen_plan_create -- plan C = A.B for n x n matrices [Algorithm 1 "Require A, B n x n"].
  *   n        matrix size (>= 1), contiguous rows (ld = n), one product per call.

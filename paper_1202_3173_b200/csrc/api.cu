@@ -43,7 +43,12 @@ struct strassen_plan {
     double *ws = nullptr;
     size_t ws_bytes = 0;
     bool own_ws = false;
-    double *stage_a = nullptr, *stage_b = nullptr, *stage_c = nullptr;
+    double *stage[2][3] = {{nullptr, nullptr, nullptr}, {nullptr, nullptr, nullptr}};   // host entry point: A, B, C copies
+    int stage_sets = 0;
+    bool host_pipeline = false;           // STRASSEN_FLAG_HOST_PIPELINE
+    cudaStream_t s_h2d = nullptr, s_cmp = nullptr, s_d2h = nullptr;
+    cudaEvent_t ev_h2d[2] = {nullptr, nullptr}, ev_cmp[2] = {nullptr, nullptr}, ev_d2h[2] = {nullptr, nullptr};
+    uint64_t host_calls = 0;
     bool timing = false;
     std::vector<TimedLaunch> pending;
     std::vector<cudaEvent_t> free_events;
@@ -237,6 +242,7 @@ strassen_plan *create(const strassen_options &o)
     }
     d.fuse_two_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) == 0;
     p->use_graph = (o.flags & STRASSEN_FLAG_CUDA_GRAPH) != 0;
+    p->host_pipeline = (o.flags & STRASSEN_FLAG_HOST_PIPELINE) != 0;
     d.sizes = level_sizes(n, cutoff);
     const size_t L = d.sizes.size() - 1;
     const bool want_auto = !o.schedule || strcmp(o.schedule, "auto") == 0;
@@ -350,44 +356,87 @@ int strassen_dgemm_host(strassen_plan *p, const double *hA, const double *hB, do
     if (!p || !hA || !hB || !hC) return fail(STRASSEN_INVALID_ARG, "plan, A, B and C must be non-NULL");
     const PlanDesc &d = p->d;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-    const size_t wa = size_t(extent_words(d.n, d.lda, d.stride_a, d.batch)) * 8;
-    const size_t wb = size_t(extent_words(d.n, d.ldb, d.stride_b, d.batch)) * 8;
-    const size_t wc = size_t(extent_words(d.n, d.ldc, d.stride_c, d.batch)) * 8;
-    if (!p->stage_a) {
-        cudaError_t e = cudaMalloc(&p->stage_a, wa);
-        if (e == cudaSuccess) e = cudaMalloc(&p->stage_b, wb);
-        if (e == cudaSuccess) e = cudaMalloc(&p->stage_c, wc);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            cudaFree(p->stage_a); cudaFree(p->stage_b); cudaFree(p->stage_c);
-            p->stage_a = p->stage_b = p->stage_c = nullptr;
-            return fail(STRASSEN_OUT_OF_MEMORY, std::string("staging buffers: ") + cudaGetErrorString(e));
+    const size_t bytes[3] = {size_t(extent_words(d.n, d.lda, d.stride_a, d.batch)) * 8,
+                             size_t(extent_words(d.n, d.ldb, d.stride_b, d.batch)) * 8,
+                             size_t(extent_words(d.n, d.ldc, d.stride_c, d.batch)) * 8};
+    if (p->stage_sets == 0) {
+        // one set of device copies; a second one (pipelined mode) if the device has room for it
+        const int want = p->host_pipeline ? 2 : 1;
+        for (int s = 0; s < want; ++s) {
+            cudaError_t e = cudaSuccess;
+            for (int m = 0; m < 3 && e == cudaSuccess; ++m) e = cudaMalloc(&p->stage[s][m], bytes[m]);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                for (int m = 0; m < 3; ++m) {
+                    cudaFree(p->stage[s][m]);
+                    p->stage[s][m] = nullptr;
+                }
+                if (s == 0) return fail(STRASSEN_OUT_OF_MEMORY, std::string("staging buffers: ") + cudaGetErrorString(e));
+                break;
+            }
+            p->stage_sets = s + 1;
+        }
+        if (p->host_pipeline) {
+            cudaError_t e = cudaStreamCreateWithFlags(&p->s_h2d, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->s_cmp, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->s_d2h, cudaStreamNonBlocking);
+            for (int s = 0; s < 2 && e == cudaSuccess; ++s) {
+                e = cudaEventCreateWithFlags(&p->ev_h2d[s], cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_cmp[s], cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_d2h[s], cudaEventDisableTiming);
+            }
+            if (e != cudaSuccess) return cuda_fail(e, "creating the streams and events of the host pipeline");
         }
     }
     const size_t row = size_t(d.n) * 8;
-    auto copy_in = [&](double *dst, int64_t ld, int64_t stride, const double *src) -> cudaError_t {
+    auto copy_in = [&](double *dst, int64_t ld, int64_t stride, const double *src, cudaStream_t st) -> cudaError_t {
         if (ld == d.n && stride == d.n * d.n)
-            return cudaMemcpyAsync(dst, src, row * size_t(d.n) * size_t(d.batch), cudaMemcpyHostToDevice, stream);
+            return cudaMemcpyAsync(dst, src, row * size_t(d.n) * size_t(d.batch), cudaMemcpyHostToDevice, st);
         for (int64_t b = 0; b < d.batch; ++b) {
             cudaError_t e = cudaMemcpy2DAsync(dst + b * stride, size_t(ld) * 8, src + b * d.n * d.n, row, row, size_t(d.n),
-                                              cudaMemcpyHostToDevice, stream);
+                                              cudaMemcpyHostToDevice, st);
             if (e != cudaSuccess) return e;
         }
         return cudaSuccess;
     };
-    cudaError_t e = copy_in(p->stage_a, d.lda, d.stride_a, hA);
-    if (e == cudaSuccess) e = copy_in(p->stage_b, d.ldb, d.stride_b, hB);
-    if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
-    const int rc = strassen_dgemm(p, p->stage_a, p->stage_b, p->stage_c, stream_v);
-    if (rc != STRASSEN_OK) return rc;
-    if (d.ldc == d.n && d.stride_c == d.n * d.n) {
-        e = cudaMemcpyAsync(hC, p->stage_c, row * size_t(d.n) * size_t(d.batch), cudaMemcpyDeviceToHost, stream);
-    } else {
-        for (int64_t b = 0; b < d.batch && e == cudaSuccess; ++b)
-            e = cudaMemcpy2DAsync(hC + b * d.n * d.n, row, p->stage_c + b * d.stride_c, size_t(d.ldc) * 8, row, size_t(d.n),
-                                  cudaMemcpyDeviceToHost, stream);
+    auto copy_out = [&](const double *src, cudaStream_t st) -> cudaError_t {
+        if (d.ldc == d.n && d.stride_c == d.n * d.n)
+            return cudaMemcpyAsync(hC, src, row * size_t(d.n) * size_t(d.batch), cudaMemcpyDeviceToHost, st);
+        for (int64_t b = 0; b < d.batch; ++b) {
+            cudaError_t e = cudaMemcpy2DAsync(hC + b * d.n * d.n, row, src + b * d.stride_c, size_t(d.ldc) * 8, row, size_t(d.n),
+                                              cudaMemcpyDeviceToHost, st);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    };
+    if (!p->host_pipeline) {
+        cudaError_t e = copy_in(p->stage[0][0], d.lda, d.stride_a, hA, stream);
+        if (e == cudaSuccess) e = copy_in(p->stage[0][1], d.ldb, d.stride_b, hB, stream);
+        if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
+        const int rc = strassen_dgemm(p, p->stage[0][0], p->stage[0][1], p->stage[0][2], stream_v);
+        if (rc != STRASSEN_OK) return rc;
+        e = copy_out(p->stage[0][2], stream);
+        if (e != cudaSuccess) return cuda_fail(e, "device-to-host copy");
+        return STRASSEN_OK;
     }
+    // Pipelined over three plan-owned streams: the input copy of this call runs beside the previous call's
+    // products and the result copy of the call before it.  An event that was never recorded does not block.
+    const int s = int(p->host_calls++ % uint64_t(p->stage_sets));
+    cudaStreamWaitEvent(p->s_h2d, p->ev_cmp[s], 0);             // the products that last read this set are done
+    cudaError_t e = copy_in(p->stage[s][0], d.lda, d.stride_a, hA, p->s_h2d);
+    if (e == cudaSuccess) e = copy_in(p->stage[s][1], d.ldb, d.stride_b, hB, p->s_h2d);
+    if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
+    cudaEventRecord(p->ev_h2d[s], p->s_h2d);
+    cudaStreamWaitEvent(p->s_cmp, p->ev_h2d[s], 0);
+    cudaStreamWaitEvent(p->s_cmp, p->ev_d2h[s], 0);             // the result copy that last read this set's C is done
+    const int rc = strassen_dgemm(p, p->stage[s][0], p->stage[s][1], p->stage[s][2], p->s_cmp);
+    if (rc != STRASSEN_OK) return rc;
+    cudaEventRecord(p->ev_cmp[s], p->s_cmp);
+    cudaStreamWaitEvent(p->s_d2h, p->ev_cmp[s], 0);
+    e = copy_out(p->stage[s][2], p->s_d2h);
     if (e != cudaSuccess) return cuda_fail(e, "device-to-host copy");
+    cudaEventRecord(p->ev_d2h[s], p->s_d2h);
+    cudaStreamWaitEvent(stream, p->ev_d2h[s], 0);               // the caller's stream sees the result
     return STRASSEN_OK;
 }
 
@@ -403,9 +452,15 @@ void strassen_plan_destroy(strassen_plan *p)
     if (p->capture_stream) cudaStreamDestroy(p->capture_stream);
     if (p->d_tab) cudaFree(p->d_tab);
     if (p->own_ws && p->ws) cudaFree(p->ws);
-    if (p->stage_a) cudaFree(p->stage_a);
-    if (p->stage_b) cudaFree(p->stage_b);
-    if (p->stage_c) cudaFree(p->stage_c);
+    for (int s = 0; s < 2; ++s) {
+        for (int m = 0; m < 3; ++m)
+            if (p->stage[s][m]) cudaFree(p->stage[s][m]);
+        if (p->ev_h2d[s]) cudaEventDestroy(p->ev_h2d[s]);
+        if (p->ev_cmp[s]) cudaEventDestroy(p->ev_cmp[s]);
+        if (p->ev_d2h[s]) cudaEventDestroy(p->ev_d2h[s]);
+    }
+    for (cudaStream_t st : {p->s_h2d, p->s_cmp, p->s_d2h})
+        if (st) cudaStreamDestroy(st);
     delete p;
 }
 

@@ -198,6 +198,22 @@ def test_host_entry_point_copies_in_and_out():
     assert np.array_equal(C.numpy(), oracle.classical(A.numpy(), B.numpy()))
 
 
+def test_host_pipeline_keeps_every_result_separate():
+    n, calls = 320, 5
+    plan = Plan(n, 80, "BB", flags=binding.STRASSEN_FLAG_HOST_PIPELINE)
+    As, Bs, Cs = [], [], []
+    for k in range(calls):
+        A, B = inputs.pair(n, "int8", 700 + 2 * k, device="cpu")
+        As.append(A.pin_memory()); Bs.append(B.pin_memory())
+        Cs.append(torch.full((n, n), float("nan"), dtype=torch.float64).pin_memory())
+    for k in range(calls):                                    # enqueue all calls back to back, no sync in between
+        plan.run_host(As[k], Bs[k], Cs[k])
+    torch.cuda.synchronize()
+    plan.close()
+    for k in range(calls):
+        assert np.array_equal(Cs[k].numpy(), oracle.classical(As[k].numpy(), Bs[k].numpy())), k
+
+
 def test_timing_split_sums_to_about_the_total():
     A, B = inputs.pair(2048, "uniform", 61, device="cuda")
     plan = Plan(2048, 512, "BB")
