@@ -110,6 +110,61 @@ def test_leading_dimensions_and_strides():
     assert bool((C[:, n:, :] == 777.0).all()) and bool((C[:, :, n:] == 777.0).all())   # nothing outside n x n
 
 
+def test_random_sizes_cutoffs_and_schedules():
+    """Seeded sweep over odd and even sizes, cutoffs and B/D strings: exact on integer inputs."""
+    rng = np.random.default_rng(2024)
+    for case in range(48):
+        n = int(rng.integers(1, 420))
+        cutoff = int(rng.integers(1, max(2, n)))
+        if n // max(cutoff, 1) > 64:            # keep the tree small: at most 6 levels
+            cutoff = max(cutoff, n // 64 + 1)
+        L = len(oracle.level_sizes(n, cutoff)) - 1
+        sched = "".join(rng.choice(list("BD"), size=L))
+        batch = int(rng.integers(1, 4))
+        check_full(n, cutoff, sched, "int8", 9000 + case, batch=batch)
+
+
+def test_pointers_that_are_only_8_byte_aligned():
+    n = 258
+    g = torch.Generator("cuda").manual_seed(77)
+    store = [torch.randint(-8, 9, (n * n + 1,), device="cuda", generator=g).double() for _ in range(2)]
+    out = torch.zeros(n * n + 1, device="cuda", dtype=torch.float64)
+    A, B, C = store[0][1:].view(n, n), store[1][1:].view(n, n), out[1:].view(n, n)     # offset by one element
+    assert A.data_ptr() % 16 == 8
+    for cutoff, sched in ((n, ""), (129, "B"), (33, "BBB"), (65, "DB")):
+        plan = Plan(n, cutoff, sched)
+        C.fill_(float("nan"))
+        binding.strassen_dgemm(plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        plan.close()
+        assert np.array_equal(C.cpu().numpy(), oracle.classical(A.cpu().numpy(), B.cpu().numpy())), (cutoff, sched)
+    assert float(out[0]) == 0.0
+
+
+@pytest.mark.parametrize("n,cutoff,sched,batch", [(771, 96, "BBB", 1), (520, 65, "DBB", 2), (1000, 125, "BDB", 1), (301, 80, "DB", 3)])
+def test_nothing_is_written_outside_the_workspace_or_c(n, cutoff, sched, batch):
+    """Guard words before and after the workspace and after C keep their pattern; padding inside the
+    workspace rows aside, every byte the library may touch is inside what it was given."""
+    plan = Plan(n, cutoff, sched, batch=batch)
+    need = plan.workspace_bytes
+    guard = 4096
+    raw = torch.full((need + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    ws = raw[guard:guard + need]
+    assert ws.data_ptr() % 256 == 0
+    binding.strassen_plan_set_workspace(plan.handle, ws.data_ptr(), need)
+    A, B = inputs.pair(n, "int8", 31 + n, device="cuda", batch=None if batch == 1 else batch)
+    cbuf = torch.full((batch * n * n + 512,), -123.0, dtype=torch.float64, device="cuda")
+    C = cbuf[:batch * n * n].view(A.shape)
+    binding.strassen_dgemm(plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    plan.close()
+    assert bool((raw[:guard] == 0x5A).all()) and bool((raw[guard + need:] == 0x5A).all())
+    assert bool((cbuf[batch * n * n:] == -123.0).all())
+    members = [(A, B, C)] if batch == 1 else [(A[b], B[b], C[b]) for b in range(batch)]
+    for a, b, c in members:
+        assert np.array_equal(c.cpu().numpy(), oracle.classical(a.cpu().numpy(), b.cpu().numpy()))
+
+
 def test_inputs_are_not_written_and_calls_repeat():
     A, B = inputs.pair(640, "uniform", 31, device="cuda")
     A0, B0 = A.clone(), B.clone()
