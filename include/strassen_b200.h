@@ -62,7 +62,8 @@ typedef enum strassen_kernel_kind {
     STRASSEN_K_FORM_ONE = 3,   /* DFS operand formation of one sub-problem j                        */
     STRASSEN_K_ACCUMULATE = 4, /* DFS fold of one Q_j into the quadrants of C                       */
     STRASSEN_K_PEEL = 5,       /* peeling fix-ups: rank-one update, last column, last row           */
-    STRASSEN_K_COUNT = 6
+    STRASSEN_K_SCALE = 6,      /* diagonal scaling passes (STRASSEN_FLAG_SCALE_*)                   */
+    STRASSEN_K_COUNT = 7
 } strassen_kernel_kind;
 
 /* Extended plan description.  Zero-initialise, then set what differs from the default. */
@@ -99,6 +100,18 @@ typedef struct strassen_options {
  * until `stream` (or the device) has been synchronised.  Without this flag everything is enqueued on
  * `stream` in order. */
 #define STRASSEN_FLAG_HOST_PIPELINE 4
+
+/* Diagonal scaling for accuracy [Section 6.1: D1 C D3 = (D1 A D2)(D2^-1 B D3)], with power-of-two
+ * diagonals so that the scaling itself is exact:
+ *   SCALE_OUTSIDE  D1, D3 bring the largest entry of every row of A and of every column of B into
+ *                  [1, 2); the error of C_ij then scales with max_k|A_ik| max_k|B_kj| instead of
+ *                  max|A| max|B| (the row/column-wise bound of Section 6.1);
+ *   SCALE_INSIDE   D2 balances column k of A against row k of B (applied before the outside scaling
+ *                  when both are set).
+ * Costs three extra passes over A and B, one over C, and 2 n^2 words of workspace (the scaled copies;
+ * counted in strassen_plan_workspace_bytes).  A and B themselves are not written. */
+#define STRASSEN_FLAG_SCALE_OUTSIDE 8
+#define STRASSEN_FLAG_SCALE_INSIDE 16
 
 /*
  * strassen_plan_create -- plan C = A.B for n x n matrices [Algorithm 1 "Require A, B n x n"].

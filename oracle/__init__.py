@@ -214,6 +214,48 @@ def lm_schedule(n: int, cutoff: int, budget_words: int, batch: int = 1, accounti
     raise ValueError("even the all-DFS schedule does not fit the budget")
 
 
+# ---------------------------------------------------------------------------
+# diagonal scaling (Section 6.1): D1 C D3 = (D1 A D2)(D2^-1 B D3) with power-of-two diagonals
+# ---------------------------------------------------------------------------
+
+def _ilog2(x):
+    """floor(log2 |x|) per element, 0 where x == 0 (exponent arithmetic, no logarithm)."""
+    x = np.abs(np.asarray(x, dtype=np.float64))
+    _, e = np.frexp(x)                      # x = m 2^e, 0.5 <= m < 1
+    return np.where(x > 0, e - 1, 0).astype(np.int64)
+
+
+def scaling_exponents(A, B, inside: bool = False, outside: bool = True):
+    """Exponents (e1, e2, e3) of D1 = diag(2^e1), D2 = diag(2^e2), D3 = diag(2^e3).
+
+    inside : balances column k of A against row k of B,
+             e2_k = floor((ilog2 max_j|B_kj| - ilog2 max_i|A_ik|) / 2);
+    outside: brings the largest entry of every row of A D2 and of every column of D2^-1 B into [1, 2),
+             e1_i = -ilog2 max_k |A_ik| 2^e2_k,  e3_j = -ilog2 max_k |B_kj| 2^-e2_k.
+    Powers of two: the scaling itself is exact, so the scaled product, unscaled, is the product."""
+    A, B = _mat(A), _mat(B)
+    n = A.shape[0]
+    e1 = np.zeros(n, dtype=np.int64)
+    e2 = np.zeros(n, dtype=np.int64)
+    e3 = np.zeros(n, dtype=np.int64)
+    if inside:
+        e2 = (_ilog2(np.abs(B).max(axis=1)) - _ilog2(np.abs(A).max(axis=0))) // 2
+    if outside:
+        e1 = -_ilog2(np.abs(np.ldexp(A, e2[None, :])).max(axis=1))
+        e3 = -_ilog2(np.abs(np.ldexp(B, -e2[:, None])).max(axis=0))
+    return e1, e2, e3
+
+
+def scaled_strassen_winograd(A, B, cutoff, schedule=None, inside: bool = False, outside: bool = True):
+    """Strassen-Winograd on the diagonally scaled operands, result scaled back (Section 6.1)."""
+    A, B = _mat(A), _mat(B)
+    e1, e2, e3 = scaling_exponents(A, B, inside, outside)
+    As = np.ldexp(A, e1[:, None] + e2[None, :])
+    Bs = np.ldexp(B, -e2[:, None] + e3[None, :])
+    Cs, cnt = strassen_winograd(As, Bs, cutoff, schedule)
+    return np.ldexp(Cs, -e1[:, None] - e3[None, :]), cnt
+
+
 def effective_gflops(n: int, seconds: float, batch: int = 1) -> float:
     """Effective GFLOPS = 2 n^3 / (seconds 10^9) (Section 5.2), times the batch size."""
     return 2.0 * n ** 3 * batch / (seconds * 1e9)

@@ -16,10 +16,12 @@ STRASSEN_OK = 0
 STRASSEN_FLAG_SINGLE_LEVEL_PASSES = 1
 STRASSEN_FLAG_CUDA_GRAPH = 2
 STRASSEN_FLAG_HOST_PIPELINE = 4
+STRASSEN_FLAG_SCALE_OUTSIDE = 8
+STRASSEN_FLAG_SCALE_INSIDE = 16
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SCHEDULE", -3: "WORKSPACE_TOO_SMALL", -4: "ALIAS",
                 -5: "MISALIGNED", -6: "CUDA_ERROR", -7: "OUT_OF_MEMORY"}
-K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_COUNT = range(7)
-KERNEL_KINDS = ("form", "gemm", "recombine", "form_one", "accumulate", "peel")
+K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_SCALE, K_COUNT = range(8)
+KERNEL_KINDS = ("form", "gemm", "recombine", "form_one", "accumulate", "peel", "scale")
 
 # every symbol the header declares: (name, restype, argtypes)
 _vp, _i64, _sz, _cp, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_char_p, ctypes.c_int

@@ -56,8 +56,8 @@ struct strassen_plan {
     cudaStream_t capture_stream = nullptr;
     cudaGraphExec_t graph_exec = nullptr;
     const void *graph_ptrs[4] = {nullptr, nullptr, nullptr, nullptr};   // A, B, C, workspace the graph was captured for
-    double acc_ms[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0};
-    int64_t launches[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0};
+    double acc_ms[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0, 0};
+    int64_t launches[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0, 0};
     int64_t launch_total = 0;
 };
 
@@ -68,6 +68,7 @@ int family(int op_kind)
 {
     if (op_kind == OP_FORM2) return STRASSEN_K_FORM;
     if (op_kind == OP_RECOMBINE2) return STRASSEN_K_RECOMBINE;
+    if (op_kind == OP_SCALE_IN || op_kind == OP_SCALE_OUT) return STRASSEN_K_SCALE;
     return op_kind;
 }
 
@@ -157,6 +158,8 @@ int enqueue_launches(strassen_plan *p, const Bases &bases, bool bases16, cudaStr
         case OP_PEEL: e = launch_peel(p->d_tab, op, bases, stream, &launched); break;
         case OP_FORM2: e = launch_form2(p->d_tab, op, bases, vec, stream, &launched); break;
         case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_SCALE_IN: e = launch_scale_in(p->d, bases, stream, &launched); break;
+        case OP_SCALE_OUT: e = launch_scale_out(p->d, bases, stream, &launched); break;
         }
         if (timed) {
             cudaEventRecord(t.stop, stream);
@@ -243,6 +246,8 @@ strassen_plan *create(const strassen_options &o)
     d.fuse_two_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) == 0;
     p->use_graph = (o.flags & STRASSEN_FLAG_CUDA_GRAPH) != 0;
     p->host_pipeline = (o.flags & STRASSEN_FLAG_HOST_PIPELINE) != 0;
+    d.scale_inside = (o.flags & STRASSEN_FLAG_SCALE_INSIDE) != 0;
+    d.scale_outside = (o.flags & STRASSEN_FLAG_SCALE_OUTSIDE) != 0;
     d.sizes = level_sizes(n, cutoff);
     const size_t L = d.sizes.size() - 1;
     const bool want_auto = !o.schedule || strcmp(o.schedule, "auto") == 0;
@@ -295,7 +300,8 @@ strassen_plan *create(const strassen_options &o)
         return nullptr;
     }
     for (const Launch &op : d.launches) {
-        const int k = launches_of(op);
+        const int k = op.kind == OP_SCALE_IN ? scale_launches(d, true) : op.kind == OP_SCALE_OUT ? scale_launches(d, false)
+                                                                                                : launches_of(op);
         p->launches[family(op.kind)] += k;
         p->launch_total += k;
     }

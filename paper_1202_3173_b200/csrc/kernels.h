@@ -81,6 +81,11 @@ constexpr int kNominalSMs = 148;   // B200; used where launches are counted with
 // Sets the shared-memory attribute of every GEMM kernel shape on the current device (idempotent).
 cudaError_t configure_gemm_kernels();
 
+// Diagonal scaling passes around the product (scale_kernels.cu).
+cudaError_t launch_scale_in(const PlanDesc &d, const Bases &bases, cudaStream_t stream, int *launched);
+cudaError_t launch_scale_out(const PlanDesc &d, const Bases &bases, cudaStream_t stream, int *launched);
+int scale_launches(const PlanDesc &d, bool in);
+
 // Kernels one replay of `op` launches (host arithmetic only; mirrors the launchers).
 int launches_of(const Launch &op);
 

@@ -247,17 +247,43 @@ std::string build_plan(PlanDesc *p)
         if (live > kMaxNodes) return "recursion tree too large for the node tables (more than 2^23 nodes)";
         p->levels.push_back(lv);
     }
+    const bool scaling = p->scale_inside || p->scale_outside;
+    if (scaling) {
+        // scaled copies of A and B (packed rows) and three int32 exponent vectors per batch member
+        p->scale_ld = round_up(p->n, 4);
+        const int64_t copy_words = round_up(p->batch * p->n * p->scale_ld, kPadWords);
+        p->scale_a_off = off;
+        p->scale_b_off = off + copy_words;
+        p->scale_exp_off = off + 2 * copy_words;
+        off = p->scale_exp_off + round_up((3 * p->batch * p->n + 1) / 2, kPadWords);
+    }
     p->ws_words = off;
 
     std::vector<Node> top(static_cast<size_t>(p->batch), Node{});
     for (int64_t b = 0; b < p->batch; ++b) {
-        top[size_t(b)].a = Operand{b * p->stride_a, int32_t(p->lda), BASE_A};
-        top[size_t(b)].b = Operand{b * p->stride_b, int32_t(p->ldb), BASE_B};
+        if (scaling) {
+            top[size_t(b)].a = ws_mat(p->scale_a_off + b * p->n * p->scale_ld, p->scale_ld);
+            top[size_t(b)].b = ws_mat(p->scale_b_off + b * p->n * p->scale_ld, p->scale_ld);
+        } else {
+            top[size_t(b)].a = Operand{b * p->stride_a, int32_t(p->lda), BASE_A};
+            top[size_t(b)].b = Operand{b * p->stride_b, int32_t(p->ldb), BASE_B};
+        }
         top[size_t(b)].c = Operand{b * p->stride_c, int32_t(p->ldc), BASE_C};
     }
     Builder bld{p, {}};
     const int64_t tab = bld.append(top);
-    if (tab >= 0) bld.build(0, tab, p->batch);
+    if (tab < 0) return bld.err;
+    if (scaling) {
+        Launch in{};
+        in.kind = OP_SCALE_IN; in.count = p->batch; in.m = p->n;
+        p->launches.push_back(in);
+    }
+    bld.build(0, tab, p->batch);
+    if (scaling && bld.err.empty()) {
+        Launch out{};
+        out.kind = OP_SCALE_OUT; out.count = p->batch; out.m = p->n;
+        p->launches.push_back(out);
+    }
     return bld.err;
 }
 

@@ -34,7 +34,9 @@ enum OpKind : int32_t {
     OP_ACCUMULATE = 4, // DFS: fold Q_j of each parent into its C quadrants
     OP_PEEL = 5,       // odd m: rank-one update, last column, last row
     OP_FORM2 = 6,      // two BFS levels at once: sums of the children and of the grandchildren
-    OP_RECOMBINE2 = 7  // two BFS levels at once: 49 grandchild products -> the parent's C
+    OP_RECOMBINE2 = 7, // two BFS levels at once: 49 grandchild products -> the parent's C
+    OP_SCALE_IN = 8,   // diagonal scaling: exponents, scaled copies of A and B in the workspace
+    OP_SCALE_OUT = 9   // diagonal scaling: C scaled back in place
 };
 
 // Regular layout of the workspace regions a two-level launch writes / reads (element offsets
@@ -78,6 +80,8 @@ struct PlanDesc {
     int64_t lda = 0, ldb = 0, ldc = 0;
     int64_t stride_a = 0, stride_b = 0, stride_c = 0;
     bool fuse_two_levels = true;    // run pairs of consecutive BFS levels as OP_FORM2 / OP_RECOMBINE2
+    bool scale_inside = false, scale_outside = false;   // diagonal scaling (Section 6.1)
+    int64_t scale_a_off = 0, scale_b_off = 0, scale_exp_off = 0, scale_ld = 0;   // workspace words / leading dimension
     std::string schedule;           // resolved, one char per level
     std::vector<int64_t> sizes;     // m_0 .. m_L
     std::vector<LevelInfo> levels;  // L entries

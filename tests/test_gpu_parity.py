@@ -269,6 +269,49 @@ def test_host_pipeline_keeps_every_result_separate():
         assert np.array_equal(Cs[k].numpy(), oracle.classical(As[k].numpy(), Bs[k].numpy())), k
 
 
+def _graded_pair(n, seed, span=24):
+    g = torch.Generator("cuda").manual_seed(seed)
+    A = (torch.rand((n, n), generator=g, device="cuda", dtype=torch.float64) * 2 - 1)
+    B = (torch.rand((n, n), generator=g, device="cuda", dtype=torch.float64) * 2 - 1)
+    ra = torch.randint(-span, span + 1, (n, 1), generator=g, device="cuda")
+    cb = torch.randint(-span, span + 1, (1, n), generator=g, device="cuda")
+    return torch.ldexp(A, ra), torch.ldexp(B, cb)
+
+
+def test_outside_scaling_meets_the_row_column_wise_bound():
+    """Section 6.1: with D1, D3 the error of C_ij scales with max_k|A_ik| max_k|B_kj|; without scaling only
+    the norm-wise bound holds.  Rows of A and columns of B spread over 2^-24 .. 2^24."""
+    n, cutoff, sched = 512, 64, "BBB"
+    A, B = _graded_pair(n, 11)
+    ref = oracle.classical(A.cpu().numpy(), B.cpu().numpy())
+    plain = run_plan(n, cutoff, sched, A, B).cpu().numpy()
+    scaled = run_plan(n, cutoff, sched, A, B, flags=binding.STRASSEN_FLAG_SCALE_OUTSIDE).cpu().numpy()
+    rows = A.abs().amax(dim=1).cpu().numpy()
+    cols = B.abs().amax(dim=0).cpu().numpy()
+    entry_bound = 4e-11 * n * rows[:, None] * cols[None, :]
+    assert np.all(np.abs(scaled - ref) <= entry_bound)
+    assert not np.all(np.abs(plain - ref) <= entry_bound)
+    assert np.abs(plain - ref).max() <= bound(n, A, B)
+    # the oracle's scaled recursion agrees to within the same bound (different summation order in the leaves)
+    want, _ = oracle.scaled_strassen_winograd(A.cpu().numpy(), B.cpu().numpy(), cutoff, sched)
+    assert np.all(np.abs(scaled - want) <= 2 * entry_bound)
+
+
+@pytest.mark.parametrize("flags", [8, 16, 24])
+def test_scaling_is_exact_on_scaled_integers(flags):
+    n, batch = 260, 2
+    g = torch.Generator("cuda").manual_seed(5)
+    A = torch.ldexp(torch.randint(-8, 9, (batch, n, n), generator=g, device="cuda").double(),
+                    torch.randint(-9, 10, (batch, n, 1), generator=g, device="cuda"))
+    B = torch.ldexp(torch.randint(-8, 9, (batch, n, n), generator=g, device="cuda").double(),
+                    torch.randint(-9, 10, (batch, 1, n), generator=g, device="cuda"))
+    A0, B0 = A.clone(), B.clone()
+    C = run_plan(n, 65, "BD", A, B, batch=batch, flags=flags)
+    assert torch.equal(A, A0) and torch.equal(B, B0)                    # inputs are scaled into copies, never in place
+    for b in range(batch):
+        assert np.array_equal(C[b].cpu().numpy(), oracle.classical(A[b].cpu().numpy(), B[b].cpu().numpy()))
+
+
 def test_timing_split_sums_to_about_the_total():
     A, B = inputs.pair(2048, "uniform", 61, device="cuda")
     plan = Plan(2048, 512, "BB")

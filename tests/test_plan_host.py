@@ -140,12 +140,12 @@ def test_launch_lists():
     single = binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES
     p = Plan(4096, 512, "BBB", flags=single)
     # (343 x 16 tiles = 37 full rounds of 148 + 12: the leaf owning the leftover runs as a second, small-tile launch)
-    assert p.launches_by_kind() == {"form": 3, "gemm": 2, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0}
+    assert p.launches_by_kind() == {"form": 3, "gemm": 2, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0}
     assert p.launch_count == 8
     p.close()
     # default: the two deepest BFS levels share one formation pass and one recombination pass
     p = Plan(4096, 512, "BBB")
-    assert p.launches_by_kind() == {"form": 2, "gemm": 2, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0}
+    assert p.launches_by_kind() == {"form": 2, "gemm": 2, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0}
     p.close()
     # DFS on top: 7 x (form_one [not for j = 0, 1], sub-tree, accumulate)
     p = Plan(16384, 512, "DBBBB", flags=single)
@@ -174,6 +174,18 @@ def test_launch_lists():
     p = Plan(300, 512, "")
     assert p.launch_count == 1 and p.workspace_bytes == 0
     p.close()
+
+
+def test_diagonal_scaling_adds_passes_and_workspace():
+    plain = Plan(4096, 512, "BBB")
+    out = Plan(4096, 512, "BBB", flags=binding.STRASSEN_FLAG_SCALE_OUTSIDE)
+    both = Plan(4096, 512, "BBB", flags=binding.STRASSEN_FLAG_SCALE_OUTSIDE | binding.STRASSEN_FLAG_SCALE_INSIDE)
+    assert out.launches_by_kind()["scale"] == 6 and both.launches_by_kind()["scale"] == 8
+    extra = out.workspace_bytes - plain.workspace_bytes
+    assert 2 * 4096 ** 2 * 8 <= extra <= 2 * 4096 ** 2 * 8 + 3 * 4096 * 4 + 1024      # two scaled copies + exponents
+    assert both.workspace_bytes == out.workspace_bytes
+    for p in (plain, out, both):
+        p.close()
 
 
 def test_batch_is_extra_live_nodes():
