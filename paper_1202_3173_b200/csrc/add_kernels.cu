@@ -44,7 +44,7 @@ __device__ __forceinline__ double *resolve(const Bases &bases, const Operand &x)
 //   T2 = A21 + A22   T3 = T2 - A11   T4 = A11 - A21   T5 = A12 - T3
 //   S2 = B12 - B11   S3 = B22 - S2   S4 = B22 - B12   S6 = S3 - B21
 // ---------------------------------------------------------------------------------------
-template <int VEC>
+template <int VEC, int RPT>
 __global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict__ parents,
                                                           const Node *__restrict__ children, Bases bases, int h,
                                                           int item0)
@@ -71,10 +71,10 @@ __global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict
         o2 = resolve(bases, kids[4].b); o3 = resolve(bases, kids[6].b);
         ldo = kids[2].b.ld;
     }
-    const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
-    T x11[ROWS_PER_THREAD], x12[ROWS_PER_THREAD], x21[ROWS_PER_THREAD], x22[ROWS_PER_THREAD];
+    const int r0 = blockIdx.y * (TY * RPT) + threadIdx.y;
+    T x11[RPT], x12[RPT], x21[RPT], x22[RPT];
 #pragma unroll
-    for (int i = 0; i < ROWS_PER_THREAD; ++i) {
+    for (int i = 0; i < RPT; ++i) {
         const int r = r0 + i * TY;
         if (r < h) {
             const double *q = X + int64_t(r) * ld + c;
@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict
         }
     }
 #pragma unroll
-    for (int i = 0; i < ROWS_PER_THREAD; ++i) {
+    for (int i = 0; i < RPT; ++i) {
         const int r = r0 + i * TY;
         if (r < h) {
             const int64_t o = int64_t(r) * ldo + c;
@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict
 //   U1 = Q0 + Q3   U2 = U1 + Q4   U3 = U1 + Q2
 //   C11 = Q0 + Q1  C12 = U3 + Q5  C21 = U2 - Q6  C22 = U2 + Q2
 // ---------------------------------------------------------------------------------------
-template <int VEC>
+template <int VEC, int RPT>
 __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__restrict__ parents,
                                                                const Node *__restrict__ children, Bases bases,
                                                                int h, int item0)
@@ -126,10 +126,10 @@ __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__res
     const Operand cc = parents[par].c;
     double *C = resolve(bases, cc);
     const int64_t ldc = cc.ld, hq = int64_t(h) * ldc;
-    const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
-    constexpr int RP = 2;   // rows per pass: 14 vectors in flight per thread
+    const int r0 = blockIdx.y * (TY * RPT) + threadIdx.y;
+    constexpr int RP = RPT < 2 ? RPT : 2;   // rows per pass: 14 vectors in flight per thread
 #pragma unroll
-    for (int pass = 0; pass < ROWS_PER_THREAD / RP; ++pass) {
+    for (int pass = 0; pass < RPT / RP; ++pass) {
         T q[RP][7];
 #pragma unroll
         for (int i = 0; i < RP; ++i) {
@@ -554,6 +554,9 @@ dim3 tile_grid(int64_t h, int vec, int64_t items)
     return dim3(unsigned((h + TX * vec - 1) / (TX * vec)), unsigned((h + TILE_ROWS - 1) / TILE_ROWS), unsigned(items));
 }
 
+// fewer than two CTAs per SM of a B200
+bool small_grid(const dim3 &g) { return int64_t(g.x) * g.y * g.z < 2 * kNominalSMs; }
+
 int chunks(int64_t items) { return int((items + MAX_Z - 1) / MAX_Z); }
 
 }  // namespace
@@ -591,12 +594,17 @@ cudaError_t launch_form(const Node *tab, const Launch &op, const Bases &bases, b
     const dim3 block(TX, TY);
     const int64_t total = op.count * 2;
     FOR_CHUNKS(total) {
-        if (vec)
-            form_bfs_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
-                                                                            bases, int(op.h), int(item0));
-        else
-            form_bfs_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
-                                                                            bases, int(op.h), int(item0));
+        const int v = vec ? 2 : 1;
+        const dim3 grid = tile_grid(op.h, v, zn);
+        const Node *par = tab + op.parent_tab, *kid = tab + op.child_tab;
+        if (small_grid(grid)) {          // too few CTAs to fill the SMs: one row per thread, four times the CTAs
+            const dim3 g1(grid.x, unsigned((op.h + TY - 1) / TY), grid.z);
+            if (vec) form_bfs_kernel<2, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+            else form_bfs_kernel<1, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+        } else {
+            if (vec) form_bfs_kernel<2, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+            else form_bfs_kernel<1, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+        }
         ++*launched;
     }
     return cudaGetLastError();
@@ -608,12 +616,17 @@ cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bas
     const dim3 block(TX, TY);
     const int64_t total = op.count;
     FOR_CHUNKS(total) {
-        if (vec)
-            recombine_bfs_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(
-                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), int(item0));
-        else
-            recombine_bfs_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(
-                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), int(item0));
+        const int v = vec ? 2 : 1;
+        const dim3 grid = tile_grid(op.h, v, zn);
+        const Node *par = tab + op.parent_tab, *kid = tab + op.child_tab;
+        if (small_grid(grid)) {
+            const dim3 g1(grid.x, unsigned((op.h + TY - 1) / TY), grid.z);
+            if (vec) recombine_bfs_kernel<2, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+            else recombine_bfs_kernel<1, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+        } else {
+            if (vec) recombine_bfs_kernel<2, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+            else recombine_bfs_kernel<1, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+        }
         ++*launched;
     }
     return cudaGetLastError();
