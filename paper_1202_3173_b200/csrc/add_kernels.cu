@@ -115,7 +115,8 @@ __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__res
 {
     using V = Vec<VEC>;
     using T = typename V::type;
-    const int par = item0 + blockIdx.z;
+    // last parent first: its products are the ones the preceding kernel wrote last, so they are still in L2
+    const int par = item0 + (gridDim.z - 1 - blockIdx.z);
     const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
     if (c >= h) return;
     const Node *kids = children + size_t(par) * 7;
@@ -341,7 +342,8 @@ __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restri
 {
     using V = Vec<VEC>;
     using T = typename V::type;
-    const int par = item0 + blockIdx.z;
+    // last parent first: its products are the ones the preceding kernel wrote last, so they are still in L2
+    const int par = item0 + (gridDim.z - 1 - blockIdx.z);
     const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
     if (c >= q) return;
     const Operand cc = parents[par].c;
