@@ -25,6 +25,7 @@ template <> struct Vec<1> {
     static __device__ __forceinline__ double add(double a, double b) { return a + b; }
     static __device__ __forceinline__ double sub(double a, double b) { return a - b; }
     static __device__ __forceinline__ double neg(double a) { return -a; }
+    static __device__ __forceinline__ double fma1(double a, double b, double v) { return fma(a, b, v); }
 };
 template <> struct Vec<2> {
     using type = double2;
@@ -34,6 +35,7 @@ template <> struct Vec<2> {
     static __device__ __forceinline__ double2 add(double2 a, double2 b) { return make_double2(a.x + b.x, a.y + b.y); }
     static __device__ __forceinline__ double2 sub(double2 a, double2 b) { return make_double2(a.x - b.x, a.y - b.y); }
     static __device__ __forceinline__ double2 neg(double2 a) { return make_double2(-a.x, -a.y); }
+    static __device__ __forceinline__ double2 fma1(double a, double2 b, double2 v) { return make_double2(fma(a, b.x, v.x), fma(a, b.y, v.y)); }
 };
 
 __device__ __forceinline__ double *resolve(const Bases &bases, const Operand &x) { return base_ptr(bases, x.base) + x.off; }
@@ -111,14 +113,27 @@ __global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict
 template <int VEC, int RPT>
 __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__restrict__ parents,
                                                                const Node *__restrict__ children, Bases bases,
-                                                               int h, int item0)
+                                                               int h, int item0, int peel)
 {
+    // peel != 0: the parent has odd size 2h + 1; the rank-one term A[r][2h] * B[2h][c] of the peeled split
+    // is added to every entry on its way out (saves a read-modify-write pass over C).
     using V = Vec<VEC>;
     using T = typename V::type;
     // last parent first: its products are the ones the preceding kernel wrote last, so they are still in L2
     const int par = item0 + (gridDim.z - 1 - blockIdx.z);
     const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
     if (c >= h) return;
+    const double *acol = nullptr;
+    int64_t lda = 0;
+    T b0 = T(), b1 = T();
+    if (peel) {
+        const Operand pa = parents[par].a, pb = parents[par].b;
+        acol = resolve(bases, pa) + 2 * h;
+        lda = pa.ld;
+        const double *brow = resolve(bases, pb) + int64_t(2 * h) * pb.ld + c;
+        b0 = V::ldk(brow);
+        b1 = V::ldk(brow + h);
+    }
     const Node *kids = children + size_t(par) * 7;
     const double *Q[7];
 #pragma unroll
@@ -148,10 +163,17 @@ __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__res
                 const T u2 = V::add(u1, q[i][4]);
                 const T u3 = V::add(u1, q[i][2]);
                 double *o = C + int64_t(r) * ldc + c;
-                V::st(o, V::add(q[i][0], q[i][1]));
-                V::st(o + h, V::add(u3, q[i][5]));
-                V::st(o + hq, V::sub(u2, q[i][6]));
-                V::st(o + hq + h, V::add(u2, q[i][2]));
+                T c11 = V::add(q[i][0], q[i][1]), c12 = V::add(u3, q[i][5]);
+                T c21 = V::sub(u2, q[i][6]), c22 = V::add(u2, q[i][2]);
+                if (peel) {
+                    const double a0 = acol[int64_t(r) * lda], a1 = acol[int64_t(r + h) * lda];
+                    c11 = V::fma1(a0, b0, c11); c12 = V::fma1(a0, b1, c12);
+                    c21 = V::fma1(a1, b0, c21); c22 = V::fma1(a1, b1, c22);
+                }
+                V::st(o, c11);
+                V::st(o + h, c12);
+                V::st(o + hq, c21);
+                V::st(o + hq + h, c22);
             }
         }
     }
@@ -209,7 +231,7 @@ __global__ void __launch_bounds__(TX *TY) form_one_kernel(const Node *__restrict
 template <int VEC>
 __global__ void __launch_bounds__(TX *TY) accumulate_kernel(const Node *__restrict__ parents,
                                                             const Node *__restrict__ children, Bases bases, int h,
-                                                            int j, int item0)
+                                                            int j, int item0, int peel)
 {
     using V = Vec<VEC>;
     using T = typename V::type;
@@ -229,7 +251,19 @@ __global__ void __launch_bounds__(TX *TY) accumulate_kernel(const Node *__restri
         double *o = C + int64_t(r) * ldc + c;
         double *c11 = o, *c12 = o + h, *c21 = o + hq, *c22 = o + hq + h;
         switch (j) {
-        case 0: V::st(c11, q); V::st(c12, q); V::st(c21, q); V::st(c22, q); break;
+        case 0:
+            if (peel) {     // odd parent: the first touch also carries the rank-one term of the peeled split
+                const Operand pa = parents[par].a, pb = parents[par].b;
+                const double *acol = resolve(bases, pa) + 2 * h;
+                const double *brow = resolve(bases, pb) + int64_t(2 * h) * pb.ld + c;
+                const double a0 = acol[int64_t(r) * pa.ld], a1 = acol[int64_t(r + h) * pa.ld];
+                const T b0 = V::ldk(brow), b1 = V::ldk(brow + h);
+                V::st(c11, V::fma1(a0, b0, q)); V::st(c12, V::fma1(a0, b1, q));
+                V::st(c21, V::fma1(a1, b0, q)); V::st(c22, V::fma1(a1, b1, q));
+            } else {
+                V::st(c11, q); V::st(c12, q); V::st(c21, q); V::st(c22, q);
+            }
+            break;
         case 1: V::st(c11, V::add(V::ldk(c11), q)); break;
         case 2: V::st(c12, V::add(V::ldk(c12), q)); V::st(c22, V::add(V::ldk(c22), q)); break;
         case 3: V::st(c12, V::add(V::ldk(c12), q)); V::st(c21, V::add(V::ldk(c21), q));
@@ -338,7 +372,7 @@ __global__ void __launch_bounds__(TX *TY) form2_kernel(const Node *__restrict__ 
 // ---------------------------------------------------------------------------------------
 template <int VEC>
 __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restrict__ parents, Bases bases, Regions2 reg,
-                                                            int q, int item0)
+                                                            int q, int item0, int peel)
 {
     using V = Vec<VEC>;
     using T = typename V::type;
@@ -351,6 +385,18 @@ __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restri
     const int64_t ldc = cc.ld, gld = reg.grand_ld;
     const double *grand = bases.p[BASE_WS] + reg.grand_q + int64_t(par) * 49 * reg.grand_mat;
     const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
+    // peel != 0: parent of odd size 4q + 1; add A[row][4q] * B[4q][col] to every entry (see recombine_bfs_kernel)
+    const double *acol = nullptr;
+    int64_t lda = 0;
+    T bv[4] = {T(), T(), T(), T()};
+    if (peel) {
+        const Operand pa = parents[par].a, pb = parents[par].b;
+        acol = resolve(bases, pa) + 4 * q;
+        lda = pa.ld;
+        const double *brow = resolve(bases, pb) + int64_t(4 * q) * pb.ld + c;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) bv[t] = V::ldk(brow + t * q);
+    }
 #pragma unroll 1
     for (int i = 0; i < ROWS_PER_THREAD; ++i) {
         const int r = r0 + i * TY;
@@ -380,10 +426,17 @@ __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restri
                 const T u3 = V::add(u1, z[2][u][v]);
                 double *o = C + (int64_t(u) * q + r) * ldc + v * q + c;     // block (u, v) of C11
                 const int64_t h = 2 * int64_t(q);
-                V::st(o, V::add(z[0][u][v], z[1][u][v]));
-                V::st(o + h, V::add(u3, z[5][u][v]));
-                V::st(o + h * ldc, V::sub(u2, z[6][u][v]));
-                V::st(o + h * ldc + h, V::add(u2, z[2][u][v]));
+                T c11 = V::add(z[0][u][v], z[1][u][v]), c12 = V::add(u3, z[5][u][v]);
+                T c21 = V::sub(u2, z[6][u][v]), c22 = V::add(u2, z[2][u][v]);
+                if (peel) {
+                    const double a0 = acol[(int64_t(u) * q + r) * lda], a1 = acol[(int64_t(u) * q + r + h) * lda];
+                    c11 = V::fma1(a0, bv[v], c11); c12 = V::fma1(a0, bv[2 + v], c12);
+                    c21 = V::fma1(a1, bv[v], c21); c22 = V::fma1(a1, bv[2 + v], c22);
+                }
+                V::st(o, c11);
+                V::st(o + h, c12);
+                V::st(o + h * ldc, c21);
+                V::st(o + h * ldc + h, c22);
             }
     }
 }
@@ -570,7 +623,7 @@ int launches_of(const Launch &op)
     case OP_RECOMBINE: return chunks(op.count);
     case OP_FORM_ONE: return chunks(op.count * ((op.j >= 2 && op.j <= 4) ? 2 : 1));
     case OP_ACCUMULATE: return chunks(op.count);
-    case OP_PEEL: return 3 * chunks(op.count);
+    case OP_PEEL: return (op.peel_fused ? 2 : 3) * chunks(op.count);
     case OP_GEMM: {
         const int rem = gemm_thin_remainder(op.m), bulk = int(op.m) - rem;
         int tiled = 0;
@@ -623,11 +676,11 @@ cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bas
         const Node *par = tab + op.parent_tab, *kid = tab + op.child_tab;
         if (small_grid(grid)) {
             const dim3 g1(grid.x, unsigned((op.h + TY - 1) / TY), grid.z);
-            if (vec) recombine_bfs_kernel<2, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
-            else recombine_bfs_kernel<1, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+            if (vec) recombine_bfs_kernel<2, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
+            else recombine_bfs_kernel<1, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
         } else {
-            if (vec) recombine_bfs_kernel<2, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
-            else recombine_bfs_kernel<1, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0));
+            if (vec) recombine_bfs_kernel<2, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
+            else recombine_bfs_kernel<1, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
         }
         ++*launched;
     }
@@ -656,10 +709,10 @@ cudaError_t launch_recombine2(const Node *tab, const Launch &op, const Bases &ba
     FOR_CHUNKS(total) {
         if (vec)
             recombine2_kernel<2><<<tile_grid(q, 2, zn), block, 0, stream>>>(tab + op.parent_tab, bases, op.reg, int(q),
-                                                                           int(item0));
+                                                                           int(item0), op.peel_fused);
         else
             recombine2_kernel<1><<<tile_grid(q, 1, zn), block, 0, stream>>>(tab + op.parent_tab, bases, op.reg, int(q),
-                                                                           int(item0));
+                                                                           int(item0), op.peel_fused);
         ++*launched;
     }
     return cudaGetLastError();
@@ -693,10 +746,10 @@ cudaError_t launch_accumulate(const Node *tab, const Launch &op, const Bases &ba
     FOR_CHUNKS(total) {
         if (vec)
             accumulate_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(
-                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), op.j, int(item0));
+                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), op.j, int(item0), op.peel_fused);
         else
             accumulate_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(
-                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), op.j, int(item0));
+                tab + op.parent_tab, tab + op.child_tab, bases, int(op.h), op.j, int(item0), op.peel_fused);
         ++*launched;
     }
     return cudaGetLastError();
@@ -737,10 +790,12 @@ cudaError_t launch_peel(const Node *tab, const Launch &op, const Bases &bases, c
     const int m = int(op.m), e = m - 1;
     const Node *nodes = tab + op.parent_tab;
     const int64_t total = op.count;
-    FOR_CHUNKS(total) {
-        peel_rank1_kernel<<<dim3((e + 63) / 64, (e + TILE_ROWS - 1) / TILE_ROWS, unsigned(zn)), dim3(64, TY), 0,
-                            stream>>>(nodes, bases, e, int(item0));
-        ++*launched;
+    if (!op.peel_fused) {       // the recombination before this launch did not carry the rank-one term
+        FOR_CHUNKS(total) {
+            peel_rank1_kernel<<<dim3((e + 63) / 64, (e + TILE_ROWS - 1) / TILE_ROWS, unsigned(zn)), dim3(64, TY), 0,
+                                stream>>>(nodes, bases, e, int(item0));
+            ++*launched;
+        }
     }
     cudaError_t err = launch_thin_cols(nodes, bases, m, m, e, 1, op.count, stream, launched);   // last column, all rows
     if (err != cudaSuccess) return err;

@@ -130,12 +130,14 @@ struct Builder {
                 build(level + 2, gtab, N2 * 7);
                 Launch r = f;
                 r.kind = OP_RECOMBINE2;
+                r.peel_fused = lv.peel;
                 p->launches.push_back(r);
             } else {
                 p->launches.push_back(f);
                 build(level + 1, ctab, N * 7);
                 Launch r = f;
                 r.kind = OP_RECOMBINE;
+                r.peel_fused = lv.peel;
                 p->launches.push_back(r);
             }
         } else {
@@ -158,12 +160,13 @@ struct Builder {
                 build(level + 1, ctab, N);
                 Launch a = f;
                 a.kind = OP_ACCUMULATE;
+                a.peel_fused = lv.peel && j == 0;
                 p->launches.push_back(a);
             }
         }
         if (lv.peel) {
             Launch x{};
-            x.kind = OP_PEEL; x.level = level; x.j = -1; x.vec_ok = 0;
+            x.kind = OP_PEEL; x.level = level; x.j = -1; x.vec_ok = 0; x.peel_fused = 1;
             x.parent_tab = tab; x.child_tab = -1; x.count = N; x.m = lv.m; x.h = h;
             p->launches.push_back(x);
         }

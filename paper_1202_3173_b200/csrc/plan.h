@@ -60,6 +60,8 @@ struct Launch {
     int64_t count;       // number of parents (leaves)
     int64_t m;           // size of the parents (leaves)
     int64_t h;           // size of the children
+    int32_t peel_fused;  // recombine / accumulate(j = 0) of an odd-size parent: also add the rank-one term
+                         // A[:, m-1] x B[m-1, :] of the peeled split; on OP_PEEL: that term is already in C
     int64_t grand_tab;   // OP_FORM2 / OP_RECOMBINE2: index of the first grandchild node
     Regions2 reg;        // OP_FORM2 / OP_RECOMBINE2 only
 };
