@@ -213,6 +213,9 @@ def main():
 
     import torch
     import torch.distributed as dist
+    from paper_1202_3173_b200 import build as _build
+    if local_rank == 0:
+        _build.ensure_built()
     from paper_1202_3173_b200 import Plan, binding, inputs
 
     if not torch.cuda.is_available():

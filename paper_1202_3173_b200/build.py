@@ -62,5 +62,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def ensure_built() -> str:
+    """Build only if the shared library is absent (used by the tests, the smoke check and the benchmark, so that a
+    checkout without build products still runs where nvcc is available)."""
+    return LIB if os.path.exists(LIB) else build()
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -24,3 +24,9 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    from paper_1202_3173_b200 import build as _build
+    _build.ensure_built()
