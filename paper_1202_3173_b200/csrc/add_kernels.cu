@@ -502,7 +502,25 @@ __global__ void __launch_bounds__(256) thin_cols_kernel(const Node *__restrict__
         const double *a0 = A + int64_t(min(rbase, rows - 1)) * nd.a.ld + k0;
         const int64_t lda = nd.a.ld;
         const int nrow = min(4, rows - rbase);
-        for (int k = lane; k < kn; k += 32) {
+        int k = lane;
+        for (; k + 32 < kn; k += 64) {              // two k per lane and pass: eight loads of A in flight
+            double av[2][4];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) av[u][i] = i < nrow ? a0[int64_t(i) * lda + k + 32 * u] : 0.0;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                double bv[NC];
+#pragma unroll
+                for (int t = 0; t < NC; ++t) bv[t] = bs[t][k + 32 * u];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int t = 0; t < NC; ++t) acc[i][t] = fma(av[u][i], bv[t], acc[i][t]);
+            }
+        }
+        for (; k < kn; k += 32) {
             double bv[NC];
 #pragma unroll
             for (int t = 0; t < NC; ++t) bv[t] = bs[t][k];
