@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(TX *TY) accumulate_kernel(const Node *__restri
 // sums of the children at each of their four quadrant positions (u, v) -- still written,
 // because the grandchildren's quadrant operands are views into them -- and from the seven
 // child operands Y_j(u, v) the four sums of each child's own children.  The parent is read
-// once instead of the children's operands being read back: 4 h^2 read + 11 h^2 written per
+// once instead of the children's operands being read back: 4 h^2 read + 10 h^2 written per
 // side instead of 11 h^2 + 11 h^2.  Same operations in the same order as two single passes.
 // ---------------------------------------------------------------------------------------
 template <int VEC>
@@ -334,11 +334,15 @@ __global__ void __launch_bounds__(TX *TY) form2_kernel(const Node *__restrict__ 
                     y[0][u][v] = x11; y[1][u][v] = x21; y[2][u][v] = s0; y[3][u][v] = s1;
                     y[4][u][v] = s2; y[5][u][v] = x22; y[6][u][v] = s3;
                 }
-                const int64_t o = (int64_t(u) * q + r) * cld + v * q + c;
-                V::st(child + o, s0);
-                V::st(child + reg.child_mat + o, s1);
-                V::st(child + 2 * reg.child_mat + o, s2);
-                V::st(child + 3 * reg.child_mat + o, s3);
+                // Below this pass the children's sums are read only as quadrant operands: X11, X12, X22 on the
+                // A side, X11, X21, X22 on the B side.  The fourth block is never read and is not written.
+                if (side == 0 ? !(u == 1 && v == 0) : !(u == 0 && v == 1)) {
+                    const int64_t o = (int64_t(u) * q + r) * cld + v * q + c;
+                    V::st(child + o, s0);
+                    V::st(child + reg.child_mat + o, s1);
+                    V::st(child + 2 * reg.child_mat + o, s2);
+                    V::st(child + 3 * reg.child_mat + o, s3);
+                }
             }
         const int64_t og = int64_t(r) * gld + c;
 #pragma unroll
