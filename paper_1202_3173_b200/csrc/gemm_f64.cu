@@ -16,6 +16,8 @@
 //   * rows padded (+4 doubles) so that the 8-byte fragment loads of a half-warp fall in 16
 //     distinct bank pairs;
 //   * each warp owns 64 x 32 of the tile: 8 x 4 DMMA accumulators of 8 x 8;
+//   * the last slab of a tile is computed strip by strip of 8 rows, and every finished strip is
+//     stored while the next one is computed, so the tile's stores drain beside tensor work;
 //   * interior slabs of 16-byte-aligned operands take a branch-free copy path; ragged edges
 //     (size not a multiple of 128 / 16) are zero-filled by cp.async's src-size operand and
 //     masked in the epilogue; operands that are only 8-byte aligned (views into matrices
@@ -46,7 +48,10 @@ template <int BM_, int BN_, int WTM_, int BK_, int STAGES_, int CTAS_> struct Cf
 };
 // Measured alternatives that did not beat CfgWide on 343 x 512^3 (33.9 TFLOP/s): 128 x 64 tiles with two
 // CTAs per SM (32.7), 32-deep slabs (33.9), 8-deep slabs (32.7), 64 x 128 tiles with 16 warps per SM (33.9).
-// What remains per tile is the drain of its 128 KB of stores (about 2.4 us of a 71 us tile at K = 512).
+// Storing the whole tile after its last slab cost 2.4 us per tile (of 71 us at K = 512); interleaved with the
+// last slab as below, and with the tile position stepped instead of divided out, 1.1 us remain.  Also measured
+// without gain: half the tile staged in shared memory for bulk-copy stores; mbarriers in place of the per-slab
+// CTA barrier (warps free to drift: per-tile cost down, steady state 1 % slower).
 using CfgWide = Cfg<128, 128, 64, 16, 4, 1>;    // 8 warps of 64 x 32; 149.5 KB of shared memory, one CTA per SM
 using CfgSmall = Cfg<64, 64, 32, 16, 4, 2>;     // 4 warps of 32 x 32; 54 KB: four times as many tiles, for launches
                                                 // whose 128 x 128 tiles would leave most SMs idle
@@ -79,16 +84,12 @@ struct TileCoord {
     int node, m0, n0;
 };
 
-template <int BM, int BN>
-__device__ __forceinline__ TileCoord tile_coord(long long t, int tiles_n, int tiles_per_node)
-{
-    TileCoord c;
-    c.node = int(t / tiles_per_node);
-    const int r = int(t - (long long)c.node * tiles_per_node);
-    c.m0 = (r / tiles_n) * BM;
-    c.n0 = (r % tiles_n) * BN;
-    return c;
-}
+// Position of a CTA in the flattened tile list: leaf and tile within the leaf.  A CTA visits tiles
+// blockIdx.x, blockIdx.x + gridDim.x, ...; stepping (node, r) by the quotient and remainder of
+// gridDim.x / tiles_per_node keeps the 64-bit division out of the loop.
+struct TileWalk {
+    int node, r;
+};
 
 // Per-thread source state of the tile currently being loaded; a and b advance slab by slab.
 struct LoadState {
@@ -125,14 +126,33 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
     const uint32_t b_dst0 = smem_base + uint32_t((A_STAGE + b_krow0 * BS + b_nc * 2) * 8);
     const bool k_ragged = (K % BK) != 0;
 
-    long long load_tile = blockIdx.x;
+    const int my_tiles = int((total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);   // the grid never exceeds total_tiles
+    const int step_node = int(gridDim.x) / tiles_per_node, step_r = int(gridDim.x) % tiles_per_node;
+    auto advance = [&](TileWalk &w) {
+        w.node += step_node;
+        w.r += step_r;
+        if (w.r >= tiles_per_node) {
+            w.r -= tiles_per_node;
+            ++w.node;
+        }
+    };
+    auto coord = [&](const TileWalk &w) {
+        TileCoord c;
+        c.node = w.node;
+        c.m0 = (w.r / tiles_n) * BM;
+        c.n0 = (w.r % tiles_n) * BN;
+        return c;
+    };
+    TileWalk load_at{int(blockIdx.x) / tiles_per_node, int(blockIdx.x) % tiles_per_node};
+    TileWalk tile_at = load_at;
+    int load_left = my_tiles;          // tiles whose loads have not been issued completely
     int load_k = 0;
     LoadState ls;
     const double *safe = reinterpret_cast<const double *>(nodes);   // valid, 16-byte aligned: for copies of 0 bytes
 
     // The node of the tile whose loads start next is fetched one slab ahead of its use, so that
     // the table read never sits between a warp and its next DMMAs.
-    TileCoord next_tc = tile_coord<BM, BN>(load_tile < total_tiles ? load_tile : 0, tiles_n, tiles_per_node);
+    TileCoord next_tc = coord(load_at);
     Operand next_a = nodes[next_tc.node].a, next_b = nodes[next_tc.node].b;
 
     auto setup_load = [&]() {
@@ -158,7 +178,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
     };
 
     auto issue_load = [&](int slot) {
-        if (load_tile < total_tiles) {
+        if (load_left > 0) {
             if (load_k == 0) setup_load();
             const uint32_t soff = uint32_t(slot * STAGE_WORDS * 8);
             if (ls.interior && !(k_ragged && load_k == ktiles - 1)) {
@@ -202,9 +222,9 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
             ls.b += B_CHUNKS * ls.b_step;
             if (++load_k == ktiles) {
                 load_k = 0;
-                load_tile += gridDim.x;
-                if (load_tile < total_tiles) {
-                    next_tc = tile_coord<BM, BN>(load_tile, tiles_n, tiles_per_node);
+                advance(load_at);
+                if (--load_left > 0) {
+                    next_tc = coord(load_at);
                     next_a = nodes[next_tc.node].a;
                     next_b = nodes[next_tc.node].b;
                 }
@@ -246,65 +266,95 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
     int slot = 0;
     load_frags(slot, 0, fa0, fb0);
 
-    for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const TileCoord tc = tile_coord<BM, BN>(tile, tiles_n, tiles_per_node);
-        const Operand c_op = nodes[tc.node].c;        // consumed after the k loop
-        for (int kt = 0; kt < ktiles; ++kt) {
-            // Invariant: every warp has passed the barrier of the previous slab, i.e. has finished
-            // reading it, so its slot may be refilled; fa0 / fb0 hold step 0 of this slab.
+    // One 16-deep slab, 4-deep step by step over all accumulators.
+    auto slab_steps = [&]() {
+        // Invariant: every warp has passed the barrier of the previous slab, i.e. has finished
+        // reading it, so its slot may be refilled; fa0 / fb0 hold step 0 of this slab.
 #pragma unroll
-            for (int kk = 0; kk < BK / 4; kk += 2) {
-                load_frags(slot, kk + 1, fa1, fb1);
-                mma_step(fa0, fb0);
-                if (kk == 0) issue_load((slot + STAGES - 1) % STAGES);
-                if (kk + 2 < BK / 4) {
-                    load_frags(slot, kk + 2, fa0, fb0);
-                } else {
-                    cp_async_wait<STAGES - 2>();      // this thread's copies of the next slab are complete
-                    __syncthreads();                  // ... and everyone's; all reads of this slab are done
-                    slot = slot + 1 == STAGES ? 0 : slot + 1;
-                    load_frags(slot, 0, fa0, fb0);
-                }
-                mma_step(fa1, fb1);
+        for (int kk = 0; kk < BK / 4; kk += 2) {
+            load_frags(slot, kk + 1, fa1, fb1);
+            mma_step(fa0, fb0);
+            if (kk == 0) issue_load((slot + STAGES - 1) % STAGES);
+            if (kk + 2 < BK / 4) {
+                load_frags(slot, kk + 2, fa0, fb0);
+            } else {
+                cp_async_wait<STAGES - 2>();      // this thread's copies of the next slab are complete
+                __syncthreads();                  // ... and everyone's; all reads of this slab are done
+                slot = slot + 1 == STAGES ? 0 : slot + 1;
+                load_frags(slot, 0, fa0, fb0);
             }
+            mma_step(fa1, fb1);
         }
-        // epilogue: this warp's 64 x 32 block of the tile
+    };
+
+    for (int t = 0; t < my_tiles; ++t, advance(tile_at)) {
+        const TileCoord tc = coord(tile_at);
+        const Operand c_op = nodes[tc.node].c;        // consumed in the last slab
+        for (int kt = 0; kt < ktiles - 1; ++kt) slab_steps();
+
+        // The last slab of the tile runs row by row of the warp's accumulators instead (all four
+        // steps of one 8-row strip, then the next strip), and each strip is stored while the next
+        // one is being computed: the tile's 128 KB of stores drain beside the DMMAs of this slab
+        // instead of holding every warp after it.
         double *C = base_ptr(bases, c_op.base) + c_op.off;
         const long long ldc = c_op.ld;
         const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((c_op.ld & 1) == 0);
         const int r0 = tc.m0 + wm * WTM + g, c0 = tc.n0 + wn * 32 + q * 2;
         double *o = C + (long long)r0 * ldc + c0;
-        if (c16 && tc.m0 + BM <= M && tc.n0 + BN <= M) {
-            // interior tile: 16-byte stores at fixed offsets from one running row pointer
+        const bool interior_out = c16 && tc.m0 + BM <= M && tc.n0 + BN <= M;
+        auto store_strip = [&](int i) {
+            double *e = o + (long long)(i * 8) * ldc;
+            if (interior_out) {
 #pragma unroll
-            for (int i = 0; i < MT; ++i) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    *reinterpret_cast<double2 *>(o + j * 8) = make_double2(acc[i][j][0], acc[i][j][1]);
-                    acc[i][j][0] = acc[i][j][1] = 0.0;
-                }
-                o += 8 * ldc;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < MT; ++i) {
+                for (int j = 0; j < 4; ++j)
+                    *reinterpret_cast<double2 *>(e + j * 8) = make_double2(acc[i][j][0], acc[i][j][1]);
+            } else {
                 const int r = r0 + i * 8;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int c = c0 + j * 8;
                     if (r < M && c < M) {
-                        double *e = o + (long long)(i * 8) * ldc + j * 8;
                         if (c + 1 < M) {
-                            if (c16) *reinterpret_cast<double2 *>(e) = make_double2(acc[i][j][0], acc[i][j][1]);
-                            else { e[0] = acc[i][j][0]; e[1] = acc[i][j][1]; }
+                            if (c16) *reinterpret_cast<double2 *>(e + j * 8) = make_double2(acc[i][j][0], acc[i][j][1]);
+                            else { e[j * 8] = acc[i][j][0]; e[j * 8 + 1] = acc[i][j][1]; }
                         } else {
-                            e[0] = acc[i][j][0];
+                            e[j * 8] = acc[i][j][0];
                         }
                     }
-                    acc[i][j][0] = acc[i][j][1] = 0.0;
                 }
             }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+        };
+        {
+            double fbL[BK / 4][4], faL[2][BK / 4];
+            const double *As = a_frag0 + slot * STAGE_WORDS, *Bs = b_frag0 + slot * STAGE_WORDS;
+#pragma unroll
+            for (int kk = 0; kk < BK / 4; ++kk) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) fbL[kk][j] = Bs[kk * 4 * BS + j * 8];
+                faL[0][kk] = As[kk * 4];
+            }
+#pragma unroll
+            for (int i = 0; i < MT; ++i) {
+                if (i + 1 < MT) {
+#pragma unroll
+                    for (int kk = 0; kk < BK / 4; ++kk) faL[(i + 1) & 1][kk] = As[(i + 1) * 8 * AS + kk * 4];
+                } else {
+                    cp_async_wait<STAGES - 2>();      // as in slab_steps: the next slab has landed,
+                    __syncthreads();                  // and every read of this one has been issued
+                    slot = slot + 1 == STAGES ? 0 : slot + 1;
+                }
+#pragma unroll
+                for (int kk = 0; kk < BK / 4; ++kk)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) dmma(acc[i][j][0], acc[i][j][1], faL[i & 1][kk], fbL[kk][j]);
+                if (i == 0) issue_load((slot + STAGES - 1) % STAGES);
+                if (i >= 1) store_strip(i - 1);
+            }
         }
+        load_frags(slot, 0, fa0, fb0);
+        store_strip(MT - 1);
     }
     cp_async_wait<0>();
 }
