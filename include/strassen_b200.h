@@ -79,10 +79,12 @@ typedef struct strassen_options {
     int64_t flags;          /* STRASSEN_FLAG_* bits; 0 = defaults                                  */
 } strassen_options;
 
-/* By default two consecutive BFS levels are formed and recombined in one pass each (the children's
- * operands are not read back and their products never written: fewer HBM bytes, same arithmetic in
- * the same order, bit-identical results).  This flag keeps one pass per level. */
+/* By default up to three consecutive BFS levels are formed and recombined in one pass each (the
+ * intermediate operands are not read back and the intermediate products never written: fewer HBM
+ * bytes, same arithmetic in the same order, bit-identical results).  SINGLE_LEVEL_PASSES keeps one
+ * pass per level, TWO_LEVEL_PASSES at most two levels per pass. */
 #define STRASSEN_FLAG_SINGLE_LEVEL_PASSES 1
+#define STRASSEN_FLAG_TWO_LEVEL_PASSES 32
 
 /* Replay the plan's launch list as one CUDA graph: the first strassen_dgemm call with a given
  * (A, B, C, workspace) captures the launches on an internal stream and instantiates the graph; that

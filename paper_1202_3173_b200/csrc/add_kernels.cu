@@ -14,7 +14,7 @@ namespace strassen {
 namespace {
 
 constexpr int TX = 64, TY = 4, ROWS_PER_THREAD = 4, TILE_ROWS = TY * ROWS_PER_THREAD;
-constexpr int MAX_Z = 32768;   // items per launch (gridDim.z limit is 65535)
+constexpr int MAX_Z = kMaxItemsPerLaunch;   // items per launch (gridDim.z limit is 65535)
 
 template <int VEC> struct Vec;
 template <> struct Vec<1> {
@@ -657,6 +657,8 @@ int launches_of(const Launch &op)
     }
     case OP_FORM2: return chunks(op.count * 2);
     case OP_RECOMBINE2: return chunks(op.count);
+    case OP_FORM3: return chunks(op.count * 2);
+    case OP_RECOMBINE3: return chunks(op.count);
     }
     return 0;
 }

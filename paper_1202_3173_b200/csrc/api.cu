@@ -66,8 +66,8 @@ namespace {
 // Kernel family (strassen_kernel_kind) a launch is counted and timed under.
 int family(int op_kind)
 {
-    if (op_kind == OP_FORM2) return STRASSEN_K_FORM;
-    if (op_kind == OP_RECOMBINE2) return STRASSEN_K_RECOMBINE;
+    if (op_kind == OP_FORM2 || op_kind == OP_FORM3) return STRASSEN_K_FORM;
+    if (op_kind == OP_RECOMBINE2 || op_kind == OP_RECOMBINE3) return STRASSEN_K_RECOMBINE;
     if (op_kind == OP_SCALE_IN || op_kind == OP_SCALE_OUT) return STRASSEN_K_SCALE;
     return op_kind;
 }
@@ -158,6 +158,8 @@ int enqueue_launches(strassen_plan *p, const Bases &bases, bool bases16, cudaStr
         case OP_PEEL: e = launch_peel(p->d_tab, op, bases, stream, &launched); break;
         case OP_FORM2: e = launch_form2(p->d_tab, op, bases, vec, stream, &launched); break;
         case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_FORM3: e = launch_form3(p->d_tab, op, bases, stream, &launched); break;
+        case OP_RECOMBINE3: e = launch_recombine3(p->d_tab, op, bases, stream, &launched); break;
         case OP_SCALE_IN: e = launch_scale_in(p->d, bases, stream, &launched); break;
         case OP_SCALE_OUT: e = launch_scale_out(p->d, bases, stream, &launched); break;
         }
@@ -243,7 +245,7 @@ strassen_plan *create(const strassen_options &o)
         delete p;
         return nullptr;
     }
-    d.fuse_two_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) == 0;
+    d.max_fused_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) ? 1 : (o.flags & STRASSEN_FLAG_TWO_LEVEL_PASSES) ? 2 : 3;
     p->use_graph = (o.flags & STRASSEN_FLAG_CUDA_GRAPH) != 0;
     p->host_pipeline = (o.flags & STRASSEN_FLAG_HOST_PIPELINE) != 0;
     d.scale_inside = (o.flags & STRASSEN_FLAG_SCALE_INSIDE) != 0;

@@ -72,16 +72,18 @@ struct Builder {
         return kids;
     }
 
-    // Levels `level` and `level + 1` run as one two-level step when both are BFS steps, the lower
-    // one is not peeled (its fix-ups need the children's own products), and the run of BFS levels
-    // starting here has even length (so that the deepest levels, which move the most bytes, pair up).
-    bool pair_starts_here(int level) const
+    // How many levels, starting at `level`, one pass forms and recombines: 1, 2 or 3.  A run of BFS
+    // levels whose lower members are not peeled (their fix-ups need the children's own products) is
+    // cut into groups of the largest allowed size from the bottom, where the bytes are; what is
+    // left over forms the group at the top of the run.
+    int group_size(int level) const
     {
-        if (!p->fuse_two_levels) return false;
-        const int L = int(p->levels.size());
+        const int L = int(p->levels.size()), g = p->max_fused_levels;
+        if (g <= 1) return 1;
         int run = 0;
         while (level + run < L && p->levels[level + run].mode == 'B' && (run == 0 || !p->levels[level + run].peel)) ++run;
-        return run >= 2 && run % 2 == 0;
+        if (run <= 1) return 1;
+        return run % g == 0 ? g : run % g;
     }
 
     // nodes of `level` are p->nodes[tab .. tab + count)
@@ -111,27 +113,46 @@ struct Builder {
             f.kind = OP_FORM; f.level = level; f.j = -1; f.vec_ok = parents_even;
             f.parent_tab = tab; f.child_tab = ctab; f.count = N; f.m = lv.m; f.h = h;
             f.grand_tab = -1;
-            if (pair_starts_here(level)) {
-                // two BFS levels in one pass: the children's sums are still written (the
-                // grandchildren's quadrant operands are views into them), their products are not
+            const int group = group_size(level);
+            if (group >= 2) {
+                // several BFS levels in one pass: the sums of the intermediate levels are still written
+                // (the operands below are views into them), their products are not
                 const LevelInfo &lv2 = p->levels[level + 1];
                 const int64_t gtab = append(bfs_children(ctab, N * 7, lv2));
                 if (gtab < 0) return;
-                f.kind = OP_FORM2;
                 f.grand_tab = gtab;
-                f.vec_ok = parents_even && (lv2.h & 1) == 0;
                 f.reg.child_t = lv.ws_off; f.reg.child_s = lv.ws_off + N * 4 * mat; f.reg.child_mat = mat;
                 f.reg.child_ld = int32_t(ldw);
                 const int64_t N2 = N * 7;
                 f.reg.grand_t = lv2.ws_off; f.reg.grand_s = lv2.ws_off + N2 * 4 * lv2.mat_words;
                 f.reg.grand_q = lv2.ws_off + N2 * 8 * lv2.mat_words; f.reg.grand_mat = lv2.mat_words;
                 f.reg.grand_ld = int32_t(lv2.ldw);
-                p->launches.push_back(f);
-                build(level + 2, gtab, N2 * 7);
-                Launch r = f;
-                r.kind = OP_RECOMBINE2;
-                r.peel_fused = lv.peel;
-                p->launches.push_back(r);
+                if (group == 2) {
+                    f.kind = OP_FORM2;
+                    f.vec_ok = parents_even && (lv2.h & 1) == 0;
+                    p->launches.push_back(f);
+                    build(level + 2, gtab, N2 * 7);
+                    Launch r = f;
+                    r.kind = OP_RECOMBINE2;
+                    r.peel_fused = lv.peel;
+                    p->launches.push_back(r);
+                } else {
+                    const LevelInfo &lv3 = p->levels[level + 2];
+                    const int64_t N3 = N2 * 7;
+                    const int64_t ggtab = append(bfs_children(gtab, N3, lv3));
+                    if (ggtab < 0) return;
+                    f.kind = OP_FORM3;
+                    f.vec_ok = 0;
+                    f.reg3.great_t = lv3.ws_off; f.reg3.great_s = lv3.ws_off + N3 * 4 * lv3.mat_words;
+                    f.reg3.great_q = lv3.ws_off + N3 * 8 * lv3.mat_words; f.reg3.great_mat = lv3.mat_words;
+                    f.reg3.great_ld = int32_t(lv3.ldw);
+                    p->launches.push_back(f);
+                    build(level + 3, ggtab, N3 * 7);
+                    Launch r = f;
+                    r.kind = OP_RECOMBINE3;
+                    r.peel_fused = lv.peel;
+                    p->launches.push_back(r);
+                }
             } else {
                 p->launches.push_back(f);
                 build(level + 1, ctab, N * 7);

@@ -36,7 +36,9 @@ enum OpKind : int32_t {
     OP_FORM2 = 6,      // two BFS levels at once: sums of the children and of the grandchildren
     OP_RECOMBINE2 = 7, // two BFS levels at once: 49 grandchild products -> the parent's C
     OP_SCALE_IN = 8,   // diagonal scaling: exponents, scaled copies of A and B in the workspace
-    OP_SCALE_OUT = 9   // diagonal scaling: C scaled back in place
+    OP_SCALE_OUT = 9,  // diagonal scaling: C scaled back in place
+    OP_FORM3 = 10,     // three BFS levels at once: sums of the children, grandchildren and great-grandchildren
+    OP_RECOMBINE3 = 11 // three BFS levels at once: 343 great-grandchild products -> the parent's C
 };
 
 // Regular layout of the workspace regions a two-level launch writes / reads (element offsets
@@ -47,6 +49,13 @@ struct Regions2 {
     int64_t grand_t, grand_s, grand_q;   // level i+2: 4 + 4 sums and 7 products per child
     int64_t grand_mat;
     int32_t child_ld, grand_ld;
+};
+
+// The third level of a three-level launch, laid out like the second.
+struct Regions3 {
+    int64_t great_t, great_s, great_q;   // level i+3: 4 + 4 sums and 7 products per grandchild
+    int64_t great_mat;
+    int32_t great_ld;
 };
 
 struct Launch {
@@ -63,7 +72,8 @@ struct Launch {
     int32_t peel_fused;  // recombine / accumulate(j = 0) of an odd-size parent: also add the rank-one term
                          // A[:, m-1] x B[m-1, :] of the peeled split; on OP_PEEL: that term is already in C
     int64_t grand_tab;   // OP_FORM2 / OP_RECOMBINE2: index of the first grandchild node
-    Regions2 reg;        // OP_FORM2 / OP_RECOMBINE2 only
+    Regions2 reg;        // OP_FORM2 / OP_RECOMBINE2 / OP_FORM3 / OP_RECOMBINE3 only
+    Regions3 reg3;       // OP_FORM3 / OP_RECOMBINE3 only
 };
 
 struct LevelInfo {
@@ -81,7 +91,7 @@ struct PlanDesc {
     int64_t n = 0, cutoff = 0, batch = 1;
     int64_t lda = 0, ldb = 0, ldc = 0;
     int64_t stride_a = 0, stride_b = 0, stride_c = 0;
-    bool fuse_two_levels = true;    // run pairs of consecutive BFS levels as OP_FORM2 / OP_RECOMBINE2
+    int max_fused_levels = 3;       // consecutive BFS levels formed / recombined by one pass: up to 3, 2 or 1
     bool scale_inside = false, scale_outside = false;   // diagonal scaling (Section 6.1)
     int64_t scale_a_off = 0, scale_b_off = 0, scale_exp_off = 0, scale_ld = 0;   // workspace words / leading dimension
     std::string schedule;           // resolved, one char per level

@@ -185,11 +185,28 @@ def test_inputs_are_not_written_and_calls_repeat():
 def test_two_level_passes_give_the_same_bits_as_single_level_passes(n, cutoff, sched, dist):
     A, B = inputs.pair(n, dist, n + 7, device="cuda")
     fused = run_plan(n, cutoff, sched, A, B)
+    two = run_plan(n, cutoff, sched, A, B, flags=binding.STRASSEN_FLAG_TWO_LEVEL_PASSES)
     single = run_plan(n, cutoff, sched, A, B, flags=binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
     assert torch.equal(fused, single)      # same operations in the same order
+    assert torch.equal(two, single)
     p1, p2 = Plan(n, cutoff, sched), Plan(n, cutoff, sched, flags=binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
     assert p1.launch_count <= p2.launch_count
     p1.close(); p2.close()
+
+
+@pytest.mark.parametrize("n,cutoff,sched,dist", [(2048, 256, "BBB", "uniform"), (1025, 128, "BBB", "normal"),
+                                                 (72, 9, "BBB", "int8"), (2064, 129, "BBBB", "uniform"),
+                                                 (1536, 24, "BBBBBB", "uniform"), (1041, 65, "DBBB", "uniform")])
+def test_three_level_passes_cover_odd_parents_ragged_tiles_and_stacked_groups(n, cutoff, sched, dist):
+    # 1025, 1041: odd size at or above the group (rank-one term inside the three-level recombination); 72: a lattice
+    # block of 9 x 9, far below one CTA tile; 2064 -> 129: a single level above a group of three with odd base;
+    # 1536 -> 24: two groups of three on top of each other
+    A, B = inputs.pair(n, dist, n + 11, device="cuda")
+    fused = run_plan(n, cutoff, sched, A, B)
+    single = run_plan(n, cutoff, sched, A, B, flags=binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
+    assert torch.equal(fused, single)
+    if n <= 1100:
+        check_full(n, cutoff, sched, dist, n + 11)
 
 
 def test_batch_with_two_level_passes():

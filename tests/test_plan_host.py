@@ -143,8 +143,13 @@ def test_launch_lists():
     assert p.launches_by_kind() == {"form": 3, "gemm": 2, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0}
     assert p.launch_count == 8
     p.close()
-    # default: the two deepest BFS levels share one formation pass and one recombination pass
+    # default: up to three BFS levels share one formation pass and one recombination pass
     p = Plan(4096, 512, "BBB")
+    assert p.launches_by_kind() == {"form": 1, "gemm": 2, "recombine": 1, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0}
+    p.close()
+    # at most two levels per pass: the two deepest levels pair up
+    two = binding.STRASSEN_FLAG_TWO_LEVEL_PASSES
+    p = Plan(4096, 512, "BBB", flags=two)
     assert p.launches_by_kind() == {"form": 2, "gemm": 2, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0}
     p.close()
     # DFS on top: 7 x (form_one [not for j = 0, 1], sub-tree, accumulate)
@@ -153,12 +158,28 @@ def test_launch_lists():
     assert k["form_one"] == 5 and k["accumulate"] == 7 and k["gemm"] == 7 and k["form"] == 28 and k["recombine"] == 28
     assert p.base_products == 7 ** 5
     p.close()
-    p = Plan(16384, 512, "DBBBB")          # four BFS levels below the DFS step: two pairs
+    p = Plan(16384, 512, "DBBBB", flags=two)          # four BFS levels below the DFS step: two pairs
     k = p.launches_by_kind()
     assert k["form"] == 14 and k["recombine"] == 14 and k["gemm"] == 7 and p.base_products == 7 ** 5
     p.close()
-    # a peeled level cannot be the lower half of a pair (its fix-ups need the children's products)
-    p = Plan(12345, 771, "BBBB")           # sizes 12345, 6172, 3086, 1543 (odd), 771: pairs (0,1) and none at (2,3)
+    p = Plan(16384, 512, "DBBBB")          # ... or one level on its own above a group of three (the bytes are at the bottom)
+    k = p.launches_by_kind()
+    assert k["form"] == 14 and k["recombine"] == 14 and k["gemm"] == 7
+    p.close()
+    p = Plan(16384, 256, "BBBBBB")         # six BFS levels: two groups of three
+    k = p.launches_by_kind()
+    assert k["form"] == 2 and k["recombine"] == 2
+    p.close()
+    p = Plan(8192, 256, "BBBBB")           # five: a pair above a group of three
+    k = p.launches_by_kind()
+    assert k["form"] == 2 and k["recombine"] == 2
+    p.close()
+    # a peeled level cannot be a lower member of a group (its fix-ups need the children's products)
+    p = Plan(12345, 771, "BBBB")           # sizes 12345, 6172, 3086, 1543 (odd), 771: group (0,1,2), then (3) alone
+    k = p.launches_by_kind()
+    assert k["form"] == 2 and k["recombine"] == 2
+    p.close()
+    p = Plan(12345, 771, "BBBB", flags=two)    # pairs: (0), (1,2), (3)
     k = p.launches_by_kind()
     assert k["form"] == 3 and k["recombine"] == 3
     p.close()
