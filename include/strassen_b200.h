@@ -144,9 +144,9 @@ strassen_plan *strassen_plan_create_ex(const strassen_options *opt);
  * All pointers must be 8-byte aligned (STRASSEN_MISALIGNED otherwise); 16-byte alignment
  * with even leading dimensions selects the vectorised paths.  Asynchronous: returns once
  * the kernels are enqueued; no host synchronisation inside, except on the first call of
- * a plan, which uploads the plan's node tables and, unless strassen_plan_set_workspace was
- * called, allocates the workspace (cudaMalloc) -- make that first call outside any stream
- * capture.  One call per plan may be in flight at a time (the workspace is shared).
+ * a plan, which uploads the plan's node tables in `stream` and waits for them (so that later
+ * calls may use any other stream) and, unless strassen_plan_set_workspace was called,
+ * allocates the workspace (cudaMalloc) -- make that first call outside any stream capture.  One call per plan may be in flight at a time (the workspace is shared).
  * The caller owns A, B, C.  NaN / Inf inputs give unspecified results (the operand sums
  * can turn Inf into NaN where the classical product would not).
  */

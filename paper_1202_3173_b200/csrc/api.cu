@@ -97,7 +97,7 @@ cudaEvent_t take_event(strassen_plan *p)
 }
 
 // First use on a device: node tables, SM count, workspace.
-int ensure_device_state(strassen_plan *p)
+int ensure_device_state(strassen_plan *p, cudaStream_t stream)
 {
     if (p->device < 0) {
         int dev = 0;
@@ -118,8 +118,15 @@ int ensure_device_state(strassen_plan *p)
         const size_t bytes = p->d.nodes.size() * sizeof(Node);
         cudaError_t e = cudaMalloc(&p->d_tab, bytes);
         if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(node tables)");
-        e = cudaMemcpy(p->d_tab, p->d.nodes.data(), bytes, cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(node tables)");
+        // In the call's own stream, then waited for: a plain cudaMemcpy from pageable memory may return while
+        // its last DMA is still queued, and a kernel in a non-blocking stream is not ordered behind it.
+        e = cudaMemcpyAsync(p->d_tab, p->d.nodes.data(), bytes, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+        if (e != cudaSuccess) {
+            cudaFree(p->d_tab);
+            p->d_tab = nullptr;
+            return cuda_fail(e, "copying the node tables to the device");
+        }
     }
     const size_t need = size_t(p->d.ws_words) * 8;
     if (need > 0 && !p->ws) {
@@ -345,9 +352,9 @@ int strassen_dgemm(strassen_plan *p, const double *A, const double *B, double *C
     const int64_t wa = extent_words(d.n, d.lda, d.stride_a, d.batch), wb = extent_words(d.n, d.ldb, d.stride_b, d.batch),
                   wc = extent_words(d.n, d.ldc, d.stride_c, d.batch);
     if (overlap(C, wc, A, wa) || overlap(C, wc, B, wb)) return fail(STRASSEN_ALIAS, "C overlaps A or B");
-    const int rc = ensure_device_state(p);
-    if (rc != STRASSEN_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int rc = ensure_device_state(p, stream);
+    if (rc != STRASSEN_OK) return rc;
     Bases bases;
     bases.p[BASE_A] = const_cast<double *>(A);
     bases.p[BASE_B] = const_cast<double *>(B);

@@ -258,6 +258,26 @@ def test_errors_on_device():
     plan.close()
 
 
+def test_first_call_on_a_side_stream_sees_its_node_tables():
+    # 137 257 nodes (6.6 MB of tables) uploaded by the first call, which is made on a non-blocking stream while
+    # another stream keeps the host-to-device copy engine busy: the product must wait for its own tables
+    n, cutoff, sched = 1024, 16, "BBBBBB"
+    A, B = inputs.pair(n, "int8", 4242, device="cuda")
+    torch.cuda.synchronize()
+    side, copier = torch.cuda.Stream(), torch.cuda.Stream()
+    host = torch.empty(1 << 28, dtype=torch.uint8).pin_memory()
+    dev = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+    with torch.cuda.stream(copier):
+        for _ in range(8):
+            dev.copy_(host, non_blocking=True)
+    plan = Plan(n, cutoff, sched)
+    with torch.cuda.stream(side):
+        C = plan(A, B)
+    torch.cuda.synchronize()
+    plan.close()
+    assert np.array_equal(C.cpu().numpy(), oracle.classical(A.cpu().numpy(), B.cpu().numpy()))
+
+
 def test_host_entry_point_copies_in_and_out():
     n = 384
     A, B = inputs.pair(n, "int8", 51, device="cpu")
