@@ -41,7 +41,7 @@ enum OpKind : int32_t {
     OP_RECOMBINE3 = 11 // three BFS levels at once: 343 great-grandchild products -> the parent's C
 };
 
-// Regular layout of the workspace regions a two-level launch writes / reads (element offsets
+// Regular layout of the workspace regions a two- or three-level launch writes / reads (element offsets
 // from the workspace base; slot s of child c sits at base + (c * slots + s) * mat).
 struct Regions2 {
     int64_t child_t, child_s;            // level i+1 operand sums: 4 per parent and side
