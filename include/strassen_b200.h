@@ -146,7 +146,9 @@ strassen_plan *strassen_plan_create_ex(const strassen_options *opt);
  * the kernels are enqueued; no host synchronisation inside, except on the first call of
  * a plan, which uploads the plan's node tables in `stream` and waits for them (so that later
  * calls may use any other stream) and, unless strassen_plan_set_workspace was called,
- * allocates the workspace (cudaMalloc) -- make that first call outside any stream capture.  One call per plan may be in flight at a time (the workspace is shared).
+ * allocates the workspace (cudaMalloc) -- make that first call outside any stream capture.
+ * A plan belongs to the device that was current on its first call (STRASSEN_INVALID_ARG on
+ * another one).  One call per plan may be in flight at a time (the workspace is shared).
  * The caller owns A, B, C.  NaN / Inf inputs give unspecified results (the operand sums
  * can turn Inf into NaN where the classical product would not).
  */

@@ -113,6 +113,16 @@ int ensure_device_state(strassen_plan *p, cudaStream_t stream)
         e = configure_gemm_kernels();       // opt-in to large dynamic shared memory, outside any capture
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute");
         p->device = dev;
+    } else {
+        // tables, workspace and staging buffers live on the device of the first call
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+        if (dev != p->device) {
+            char buf[128];
+            snprintf(buf, sizeof buf, "the plan was first used on device %d; the current device is %d", p->device, dev);
+            return fail(STRASSEN_INVALID_ARG, buf);
+        }
     }
     if (!p->d_tab) {
         const size_t bytes = p->d.nodes.size() * sizeof(Node);
