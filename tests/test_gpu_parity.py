@@ -258,6 +258,17 @@ def test_errors_on_device():
     plan.close()
 
 
+@pytest.mark.parametrize("n,cutoff,sched,flags", [(2048, 16, "BBBBBBB", 0), (2048, 16, "BBBBBBB", 1), (1024, 8, "BBBBBBB", 32)])
+def test_item_lists_longer_than_one_launch_covers(n, cutoff, sched, flags):
+    # 7^6 = 117 649 parents at the deepest level and 7^7 = 823 543 leaves: the streaming kernels and the thin
+    # products (8 x 8 leaves are all remainder) cut their item lists into launches of at most 32 768 items
+    if _free_bytes() < 12 * GB:
+        pytest.skip("needs 8 GB")
+    A, B = inputs.pair(n, "int8", 900 + n + flags, device="cuda")
+    C = run_plan(n, cutoff, sched, A, B, flags=flags)
+    assert np.array_equal(C.cpu().numpy(), oracle.classical(A.cpu().numpy(), B.cpu().numpy()))
+
+
 def test_first_call_on_a_side_stream_sees_its_node_tables():
     # 137 257 nodes (6.6 MB of tables) uploaded by the first call, which is made on a non-blocking stream while
     # another stream keeps the host-to-device copy engine busy: the product must wait for its own tables
