@@ -650,8 +650,8 @@ int launches_of(const Launch &op)
         const int rem = gemm_thin_remainder(op.m), bulk = int(op.m) - rem;
         int tiled = 0;
         if (bulk > 0) {
-            const GemmSplit split = gemm_split(bulk, op.count, kNominalSMs);
-            tiled = (!split.all_small && split.wide_leaves < op.count) ? 2 : 1;
+            GemmRegion regions[4];
+            tiled = gemm_regions(bulk, op.count, kNominalSMs, regions);
         }
         return tiled + (rem ? chunks(op.count) * (bulk > 0 ? 2 : 1) : 0);
     }

@@ -97,7 +97,7 @@ struct LoadState {
     const double *b;        // element (k0 + krow0, n0 + 2 nc) of B
     long long a_step;       // A_ROWS_STEP rows of A
     long long b_step;       // B_KROWS_STEP rows of B
-    int a_rows_ok;          // bit i: row m0 + row0 + A_ROWS_STEP i < M
+    int a_rows_ok;          // bit i: row m0 + row0 + A_ROWS_STEP i lies inside the block
     int b_cols;             // valid columns of this thread's B chunk: 0, 1 or 2
     bool a16, b16;          // 16-byte copies legal
     bool interior;          // all rows / columns valid and both operands 16-byte aligned
@@ -105,10 +105,10 @@ struct LoadState {
 
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, C::CTAS)
-gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int tiles_n, int tiles_per_node, int ktiles,
+gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, GemmRegion reg, int K, int tiles_n, int tiles_per_node, int ktiles,
                 long long total_tiles)
 {
-    // M: extent of the output block computed here (rows and columns); K: inner dimension.
+    // reg: the block of every leaf's output computed here (tiles are counted from its corner); K: inner dimension.
     constexpr int BM = C::BM, BN = C::BN, WTM = C::WTM, MT = C::MT, BK = C::BK, AS = C::AS, BS = C::BS, STAGES = C::STAGES, STAGE_WORDS = C::STAGE_WORDS;
     constexpr int A_STAGE = C::A_STAGE, A_CHUNKS = C::A_CHUNKS, A_ROWS_STEP = C::A_ROWS_STEP, A_KCHUNKS = C::A_KCHUNKS;
     constexpr int B_CHUNKS = C::B_CHUNKS, B_KROWS_STEP = C::B_KROWS_STEP;
@@ -139,8 +139,8 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
     auto coord = [&](const TileWalk &w) {
         TileCoord c;
         c.node = w.node;
-        c.m0 = (w.r / tiles_n) * BM;
-        c.n0 = (w.r % tiles_n) * BN;
+        c.m0 = reg.row0 + (w.r / tiles_n) * BM;
+        c.n0 = reg.col0 + (w.r % tiles_n) * BN;
         return c;
     };
     TileWalk load_at{int(blockIdx.x) / tiles_per_node, int(blockIdx.x) % tiles_per_node};
@@ -169,12 +169,12 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
         ls.a_rows_ok = 0;
 #pragma unroll
         for (int i = 0; i < A_CHUNKS; ++i)
-            if (tc.m0 + a_row0 + A_ROWS_STEP * i < M) ls.a_rows_ok |= 1 << i;
+            if (tc.m0 + a_row0 + A_ROWS_STEP * i < reg.row_end) ls.a_rows_ok |= 1 << i;
         ls.a = A + (long long)(tc.m0 + a_row0) * nd.a.ld + a_kc * 2;
         const int col = tc.n0 + b_nc * 2;
-        ls.b_cols = max(0, min(2, M - col));
+        ls.b_cols = max(0, min(2, reg.col_end - col));
         ls.b = B + (long long)b_krow0 * nd.b.ld + col;
-        ls.interior = ls.a16 && ls.b16 && tc.m0 + BM <= M && tc.n0 + BN <= M;
+        ls.interior = ls.a16 && ls.b16 && tc.m0 + BM <= reg.row_end && tc.n0 + BN <= reg.col_end;
     };
 
     auto issue_load = [&](int slot) {
@@ -301,7 +301,7 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
         const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((c_op.ld & 1) == 0);
         const int r0 = tc.m0 + wm * WTM + g, c0 = tc.n0 + wn * 32 + q * 2;
         double *o = C + (long long)r0 * ldc + c0;
-        const bool interior_out = c16 && tc.m0 + BM <= M && tc.n0 + BN <= M;
+        const bool interior_out = c16 && tc.m0 + BM <= reg.row_end && tc.n0 + BN <= reg.col_end;
         auto store_strip = [&](int i) {
             double *e = o + (long long)(i * 8) * ldc;
             if (interior_out) {
@@ -313,8 +313,8 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, int M, int K, int t
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int c = c0 + j * 8;
-                    if (r < M && c < M) {
-                        if (c + 1 < M) {
+                    if (r < reg.row_end && c < reg.col_end) {
+                        if (c + 1 < reg.col_end) {
                             if (c16) *reinterpret_cast<double2 *>(e + j * 8) = make_double2(acc[i][j][0], acc[i][j][1]);
                             else { e[j * 8] = acc[i][j][0]; e[j * 8 + 1] = acc[i][j][1]; }
                         } else {
@@ -372,8 +372,7 @@ cudaError_t configure_gemm_kernels();
 namespace {
 
 template <class C>
-cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, int K, long long count, int sm_count,
-                       cudaStream_t stream)
+cudaError_t launch_cfg(const Node *nodes, const Bases &bases, const GemmRegion &reg, int K, int sm_count, cudaStream_t stream)
 {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -382,13 +381,13 @@ cudaError_t launch_cfg(const Node *nodes, const Bases &bases, int M, int K, long
         e = configure_gemm_kernels();
         if (e != cudaSuccess) return e;
     }
-    const int tiles_m = (M + C::BM - 1) / C::BM, tiles_n = (M + C::BN - 1) / C::BN;
+    const int tiles_m = (reg.row_end - reg.row0 + C::BM - 1) / C::BM, tiles_n = (reg.col_end - reg.col0 + C::BN - 1) / C::BN;
     const int tiles_per_node = tiles_m * tiles_n;
     const int ktiles = (K + C::BK - 1) / C::BK;
-    const long long total = (long long)tiles_per_node * count;
+    const long long total = (long long)tiles_per_node * reg.leaves;
     const long long slots = (long long)sm_count * C::CTAS;
     const int grid = int(total < slots ? total : slots);
-    gemm_f64_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(nodes, bases, M, K, tiles_n, tiles_per_node, ktiles, total);
+    gemm_f64_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(nodes + reg.first, bases, reg, K, tiles_n, tiles_per_node, ktiles, total);
     return cudaGetLastError();
 }
 
@@ -417,18 +416,12 @@ cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, i
     const Node *nodes = tab + op.parent_tab;
     cudaError_t err = cudaSuccess;
     if (M > 0) {
-        const GemmSplit split = gemm_split(M, op.count, sm_count);
-        if (split.all_small) {
+        GemmRegion regions[4];
+        const int nreg = gemm_regions(M, op.count, sm_count, regions);
+        for (int i = 0; i < nreg && err == cudaSuccess; ++i) {
             ++*launched;
-            err = launch_cfg<CfgSmall>(nodes, bases, M, K, op.count, sm_count, stream);
-        } else {
-            ++*launched;
-            err = launch_cfg<CfgWide>(nodes, bases, M, K, split.wide_leaves, sm_count, stream);
-            if (err == cudaSuccess && split.wide_leaves < op.count) {
-                ++*launched;
-                err = launch_cfg<CfgSmall>(nodes + split.wide_leaves, bases, M, K, op.count - split.wide_leaves, sm_count,
-                                           stream);
-            }
+            err = regions[i].small ? launch_cfg<CfgSmall>(nodes, bases, regions[i], K, sm_count, stream)
+                                   : launch_cfg<CfgWide>(nodes, bases, regions[i], K, sm_count, stream);
         }
         if (err != cudaSuccess) return err;
     }

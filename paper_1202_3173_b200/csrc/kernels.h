@@ -82,6 +82,49 @@ inline GemmSplit gemm_split(int64_t M, int64_t count, int sms)
     }
     return GemmSplit{false, wide_leaves};
 }
+
+// One tiled launch of the base products: the block [row0, row_end) x [col0, col_end) of C for the leaves
+// [first, first + leaves), on the 128 x 128 tiling or the 64 x 64 one.
+struct GemmRegion {
+    bool small;
+    int row0, col0, row_end, col_end;
+    int64_t first, leaves;
+};
+// The tiled launches that cover the M x M output of `count` leaves.  Where M ends 1..64 past a multiple of
+// 128, the 128 x 128 tiling would spend whole tiles on that margin; the leaves on that tiling then take the
+// margin as a right and a bottom strip of 64 x 64 tiles (worth it from a few full rounds of strip tiles on).
+// Writes at most 4 entries to `out` and returns their number.
+inline int gemm_regions(int64_t M64, int64_t count, int sms, GemmRegion *out)
+{
+    const int M = int(M64);
+    int k = 0;
+    const int margin = M % 128, bulk = M - margin;
+    bool strips = false;
+    if (margin >= 1 && margin <= 64 && bulk > 0) {
+        // rounds x tile cost in eighteenths of a 128 x 128 tile time: such a tile alone on an SM costs 18, a
+        // 64 x 64 tile beside another one 10 (two per SM, a little slower per flop), a launch's ramp 2
+        const auto rounds = [](int64_t tiles, int64_t slots) { return (tiles + slots - 1) / slots; };
+        const int64_t tw = (M + 127) / 128, ts = (M + 63) / 64, tb = bulk / 128, strip_tiles = 2 * (bulk / 64) + 1;
+        const int64_t whole_wide = rounds(tw * tw * count, sms) * 18;
+        const int64_t whole_small = rounds(ts * ts * count, 2 * sms) * 10 + 2;
+        const int64_t with_strips = rounds(tb * tb * count, sms) * 18 + rounds(strip_tiles * count, 2 * sms) * 10 + 4;
+        strips = strip_tiles * count >= 4 * int64_t(sms) && with_strips < whole_wide && with_strips < whole_small;
+    }
+    if (!strips && gemm_split(M, count, sms).all_small) {
+        out[k++] = GemmRegion{true, 0, 0, M, M, 0, count};
+        return k;
+    }
+    const int wide_extent = strips ? bulk : M;
+    const GemmSplit split = gemm_split(wide_extent, count, sms);       // which leaves fill whole rounds of large tiles
+    const int64_t wide_leaves = split.all_small ? count : split.wide_leaves;
+    out[k++] = GemmRegion{false, 0, 0, wide_extent, wide_extent, 0, wide_leaves};
+    if (strips) {
+        out[k++] = GemmRegion{true, 0, bulk, bulk, M, 0, wide_leaves};     // right strip
+        out[k++] = GemmRegion{true, bulk, 0, M, M, 0, wide_leaves};        // bottom strip with the corner
+    }
+    if (wide_leaves < count) out[k++] = GemmRegion{true, 0, 0, M, M, wide_leaves, count - wide_leaves};
+    return k;
+}
 constexpr int kNominalSMs = 148;   // B200; used where launches are counted without a device at hand
 
 // Sets the shared-memory attribute of every GEMM kernel shape on the current device (idempotent).

@@ -37,6 +37,24 @@ def test_base_product_thin_remainders(n):
     check_full(n, n, "", "normal", 301 + n, batch=3)
 
 
+@pytest.mark.parametrize("n,cutoff,sched,batch", [(4480, 560, "BBB", 1), (2400, 300, "BBB", 2), (4481, 560, "BBB", 1)])
+def test_base_product_margin_strips(n, cutoff, sched, batch):
+    # a base size 1..64 past a multiple of 128 with hundreds of leaves: 128 x 128 tiles over the multiple, a right
+    # and a bottom strip of 64 x 64 tiles over the margin (560 = 512 + 48, 300 = 256 + 44; 4481: leaves that are
+    # views with an odd leading dimension)
+    p = Plan(n, cutoff, sched, batch=batch)
+    assert p.launches_by_kind()["gemm"] >= 3
+    p.close()
+    members = (0,) if batch == 1 else (0, batch - 1)
+    check_sampled(n, cutoff, sched, "int8", 640 + n, batch=batch, members=members)
+    check_sampled(n, cutoff, sched, "uniform", 641 + n, batch=batch, members=members)
+
+
+@pytest.mark.parametrize("n,batch,dist", [(300, 70, "int8"), (192, 100, "uniform"), (560, 40, "int8")])
+def test_base_product_batches_with_a_margin(n, batch, dist):
+    check_full(n, n, "", dist, 650 + n, batch=batch)
+
+
 def test_base_product_split_between_tile_shapes():
     # 5 x 30 x 30... enough 128-tiles for >= 4 full rounds of 148 plus a short tail that moves to 64 x 64 tiles
     check_full(512, 512, "", "int8", 77, batch=38)       # 608 tiles = 4 rounds + 16
