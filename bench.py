@@ -43,7 +43,7 @@ UNIT = "GFLOP/s"
 
 # DRAM bytes (read + write) of the dominant kernel's launch from one ncu capture, per workload
 # (profiles/gemm_f64_kernel_343x512.md); None where no capture of that exact launch exists.
-GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.127e9, "gemm512x343": 2.127e9}
+GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.125e9, "gemm512x343": 2.125e9}
 
 # FP64 arithmetic peak from unit counts and clocks: 148 SMs x 64 FP64 FMA lanes x 2 flop x 1.965 GHz
 FP64_PEAK_NOMINAL_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
@@ -344,15 +344,19 @@ def main():
         del Cc
 
     tuned = None
-    if not args.no_autotune and batch * n * n * 8 * 3 < 20e9:
+    if not args.no_autotune:
         # the paper tunes every point to the best interleaving and number of Strassen steps (Section 5.4);
         # reported beside the prescribed configuration, never instead of it
         try:
-            ws_budget = max(plan.workspace_bytes, int(min(40e9, torch.cuda.mem_get_info()[0] - 2e9)))
-            ws = torch.empty(ws_budget, dtype=torch.uint8, device=dev)
-            Ct = torch.empty_like(A)
-            best, log = binding.strassen_autotune(n, A.data_ptr(), B.data_ptr(), Ct.data_ptr(), ws.data_ptr(), ws_budget,
-                                                  stream.cuda_stream, batch, 256, 3, 60.0)
+            if batch * n * n * 8 * 3 < 20e9:
+                ws_budget = max(plan.workspace_bytes, int(min(40e9, torch.cuda.mem_get_info()[0] - 2e9)))
+                ws = torch.empty(ws_budget, dtype=torch.uint8, device=dev)
+                Ct = torch.empty_like(A)
+            else:       # no room for a second workspace and result: the plan's own workspace and C serve the search
+                ws_budget, ws, Ct = plan.workspace_bytes, plan.workspace, C
+            best, log = binding.strassen_autotune(n, A.data_ptr(), B.data_ptr(), Ct.data_ptr(),
+                                                  ws.data_ptr() if ws is not None else 0, ws_budget,
+                                                  stream.cuda_stream, batch, 256, 3 if n < 20000 else 1, 60.0)
             tuned = dict(best, candidates=len(log), gflops=2.0 * n ** 3 * batch / (best["ms"] * 1e-3) / 1e9,
                          workspace_budget_bytes=ws_budget)
             del ws, Ct

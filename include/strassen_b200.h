@@ -217,8 +217,10 @@ int strassen_plan_get_timings(strassen_plan *plan, double *ms_out /* [STRASSEN_K
  * Candidates: for every step count L whose base size floor(n / 2^L) is >= min_base, every string of
  * L characters over {B, D} whose workspace fits `workspace_bytes`.  Each candidate runs once to warm
  * up and `repetitions` more times on `stream`, timed with CUDA events; the fastest run counts.  The
- * search stops early after `max_seconds`.  On return *best holds the winner, `log` (if given) the
- * first log_capacity candidates in search order, and C the product computed with the winner's plan
+ * candidates are tried in the order of a cost model (DMMA time of the base products' tiling + HBM
+ * bytes of the passes + launches), most promising first, and the search stops after `max_seconds`.
+ * On return *best holds the winner, `log` (if given) the first log_capacity candidates in the order
+ * they were tried, and C the product computed with the winner's plan
  * (the stream is synchronised).  A, B, C: device pointers as for strassen_dgemm with ld = n; the
  * caller owns them and the workspace.  Synchronous; allocates only the per-plan node tables.
  */
@@ -239,6 +241,7 @@ typedef struct strassen_tune_entry {
     int levels;
     char schedule[36];
     double ms;                 /* best measured time of one product                          */
+    double model_ms;           /* the cost model's estimate that ordered the search          */
 } strassen_tune_entry;
 
 int strassen_autotune(const strassen_tune_request *request, strassen_tune_entry *best, strassen_tune_entry *log,

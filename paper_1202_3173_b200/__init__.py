@@ -57,6 +57,11 @@ class Plan:
         return binding.strassen_plan_workspace_bytes(self._h)
 
     @property
+    def workspace(self):
+        """The torch tensor holding the workspace (None before the first call or for plans without one)."""
+        return self._ws
+
+    @property
     def launch_count(self):
         return binding.strassen_plan_launch_count(self._h)
 

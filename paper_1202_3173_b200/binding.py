@@ -42,10 +42,12 @@ class strassen_tune_request(ctypes.Structure):
 
 
 class strassen_tune_entry(ctypes.Structure):
-    _fields_ = [("cutoff", _i64), ("levels", _int), ("schedule", ctypes.c_char * 36), ("ms", ctypes.c_double)]
+    _fields_ = [("cutoff", _i64), ("levels", _int), ("schedule", ctypes.c_char * 36), ("ms", ctypes.c_double),
+                ("model_ms", ctypes.c_double)]
 
     def as_dict(self):
-        return {"cutoff": int(self.cutoff), "levels": int(self.levels), "schedule": self.schedule.decode(), "ms": float(self.ms)}
+        return {"cutoff": int(self.cutoff), "levels": int(self.levels), "schedule": self.schedule.decode(), "ms": float(self.ms),
+                "model_ms": float(self.model_ms)}
 
 
 SYMBOLS = [

@@ -72,19 +72,7 @@ struct Builder {
         return kids;
     }
 
-    // How many levels, starting at `level`, one pass forms and recombines: 1, 2 or 3.  A run of BFS
-    // levels whose lower members are not peeled (their fix-ups need the children's own products) is
-    // cut into groups of the largest allowed size from the bottom, where the bytes are; what is
-    // left over forms the group at the top of the run.
-    int group_size(int level) const
-    {
-        const int L = int(p->levels.size()), g = p->max_fused_levels;
-        if (g <= 1) return 1;
-        int run = 0;
-        while (level + run < L && p->levels[level + run].mode == 'B' && (run == 0 || !p->levels[level + run].peel)) ++run;
-        if (run <= 1) return 1;
-        return run % g == 0 ? g : run % g;
-    }
+    int group_size(int level) const { return fused_group_size(p->sizes, p->schedule, level, p->max_fused_levels); }
 
     // nodes of `level` are p->nodes[tab .. tab + count)
     void build(int level, int64_t tab, int64_t count)
@@ -195,6 +183,19 @@ struct Builder {
 };
 
 }  // namespace
+
+// A run of BFS levels whose lower members are not peeled (their fix-ups need the children's own
+// products) is cut into groups of the largest allowed size from the bottom, where the bytes are;
+// what is left over forms the group at the top of the run.
+int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused)
+{
+    const int L = int(sched.size());
+    if (max_fused <= 1 || level >= L || sched[level] != 'B') return 1;
+    int run = 0;
+    while (level + run < L && sched[level + run] == 'B' && (run == 0 || (sizes[level + run] & 1) == 0)) ++run;
+    if (run <= 1) return 1;
+    return run % max_fused == 0 ? max_fused : run % max_fused;
+}
 
 std::vector<int64_t> level_sizes(int64_t n, int64_t cutoff)
 {

@@ -102,6 +102,10 @@ struct PlanDesc {
     std::vector<Launch> launches;   // replayed in order by strassen_dgemm
 };
 
+// How many levels, starting at `level`, one pass forms and recombines (1 .. max_fused) under schedule
+// `sched` with level sizes `sizes`; 1 for a DFS level.
+int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused);
+
 // Level sizes m_0 = n, m_{i+1} = floor(m_i / 2) while m_i > cutoff.
 std::vector<int64_t> level_sizes(int64_t n, int64_t cutoff);
 

@@ -1,10 +1,12 @@
 // strassen_autotune: measured choice of the number of Strassen steps and of the BFS/DFS
 // interleaving (Section 5.4: every point of the paper's plot is tuned to the best interleaving
 // pattern and the best total number of Strassen steps).  Brute force over the candidates that fit
-// the caller's workspace, timed with CUDA events on the caller's stream.
+// the caller's workspace, timed with CUDA events on the caller's stream, in the order of a cost
+// model so that a time limit cuts off the unlikely ones.
 #include "strassen_b200.h"
 
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
 #include <string>
 #include <vector>
@@ -22,6 +24,63 @@ int tune_fail(int status, const std::string &msg)
 {
     set_last_error(msg.c_str());
     return status;
+}
+
+// Estimate of one product's time from the quantities the kernels are bound by (measured on B200): the base
+// products at the DMMA rate of their tiling, everything else as HBM bytes, a few microseconds per launch.
+// Only used to decide which candidates are tried first; the choice itself is by measurement.
+double model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch)
+{
+    const int L = int(sched.size());
+    const double hbm = 6.2e12, launch_us = 3.0;
+    double bytes = 0.0, launches = 0.0, visits = double(batch), sequential = 1.0;   // node visits at the current level
+    for (int level = 0; level < L;) {
+        const double m = double(sizes[level]), h = double(sizes[level + 1]);
+        if (sizes[level] & 1) {
+            bytes += visits * 2.0 * m * m * 8.0;      // last column and last row: each reads one operand in full
+            launches += 2.0 * sequential;
+        }
+        if (sched[level] == 'D') {
+            bytes += visits * 57.0 * h * h * 8.0;     // 30 h^2 to form the operands one at a time, 27 h^2 to fold the products
+            launches += 12.0 * sequential;
+            visits *= 7.0;
+            sequential *= 7.0;
+            ++level;
+            continue;
+        }
+        const int g = fused_group_size(sizes, sched, level, 3);
+        const double words = g == 1 ? 27.0 : g == 2 ? 28.0 + 16.25 : 49.0 + 25.5;    // per parent, in h^2 of its children
+        bytes += visits * words * h * h * 8.0;
+        launches += 2.0 * sequential;
+        for (int i = 0; i < g; ++i) visits *= 7.0;
+        level += g;
+    }
+    const int64_t b = sizes[L];
+    const double leaves = visits, kp = double((b + 15) / 16 * 16);
+    const int rem = gemm_thin_remainder(b);
+    double us = 0.0;
+    if (b - rem > 0) {
+        GemmRegion regions[4];
+        const int64_t count = leaves > 4.0e9 ? int64_t(4e9) : int64_t(leaves);
+        const int nreg = gemm_regions(b - rem, count, kNominalSMs, regions);
+        const double wide_tile_us = kp / 16.0 * 2.147 + 1.1;      // one 128 x 128 tile on an SM: per 16-deep slab and per tile
+        for (int i = 0; i < nreg; ++i) {
+            const GemmRegion &r = regions[i];
+            const int t = r.small ? 64 : 128;
+            const double tiles = double((r.row_end - r.row0 + t - 1) / t) * double((r.col_end - r.col0 + t - 1) / t) * double(r.leaves);
+            const double slots = r.small ? 2.0 * kNominalSMs : double(kNominalSMs);
+            const double tile_us = r.small ? wide_tile_us * 0.5 / 0.88 : wide_tile_us;
+            double rounds = tiles / sequential / slots;          // per launch: a DFS level above runs its sub-trees one by one
+            if (rounds < 1.0) rounds = 1.0;
+            us += rounds * tile_us * sequential;
+            launches += sequential;
+        }
+    }
+    if (rem) {
+        bytes += leaves * 2.0 * double(b) * double(b) * 8.0;
+        launches += 2.0 * sequential;
+    }
+    return us * 1e-3 + bytes / hbm * 1e3 + launches * launch_us * 1e-3;
 }
 
 }  // namespace
@@ -53,18 +112,37 @@ extern "C" int strassen_autotune(const strassen_tune_request *req, strassen_tune
     // L Strassen steps <=> cutoff = size of level L (recursion continues while size > cutoff)
     std::vector<int64_t> sizes{n};
     while (sizes.back() / 2 >= min_base && sizes.size() <= 10) sizes.push_back(sizes.back() / 2);
-    for (size_t L = 0; L < sizes.size() && !out_of_time && status == STRASSEN_OK; ++L) {
-        const int64_t cutoff = sizes[L];
-        for (unsigned mask = 0; mask < (1u << L) && !out_of_time; ++mask) {
+    struct Candidate {
+        int64_t cutoff;
+        std::string sched;
+        double model;
+    };
+    std::vector<Candidate> candidates;
+    for (size_t L = 0; L < sizes.size(); ++L) {
+        const std::vector<int64_t> chain(sizes.begin(), sizes.begin() + L + 1);
+        for (unsigned mask = 0; mask < (1u << L); ++mask) {
             std::string sched(L, 'B');
             for (size_t i = 0; i < L; ++i)
                 if (mask >> i & 1) sched[i] = 'D';
+            const int64_t words = actual_workspace_words(chain, sched, batch);
+            if (words < 0 || size_t(words) > req->workspace_bytes / 8) continue;       // does not fit the workspace
+            candidates.push_back(Candidate{sizes[L], sched, model_ms(chain, sched, batch)});
+        }
+    }
+    // most promising first, so that a search cut short by max_seconds has seen the likely winners
+    std::stable_sort(candidates.begin(), candidates.end(), [](const Candidate &a, const Candidate &b) { return a.model < b.model; });
+    for (const Candidate &cand : candidates) {
+        if (out_of_time || status != STRASSEN_OK) break;
+        {
+            const int64_t cutoff = cand.cutoff;
+            const std::string &sched = cand.sched;
+            const size_t L = sched.size();
             strassen_options o;
             memset(&o, 0, sizeof o);
             o.n = n; o.cutoff = cutoff; o.schedule = sched.c_str(); o.batch = batch;
             o.workspace_budget_bytes = req->workspace_bytes ? req->workspace_bytes : 1;   // explicit schedules are checked against it
             strassen_plan *p = strassen_plan_create_ex(&o);
-            if (!p) continue;                                   // does not fit the workspace (or the node tables)
+            if (!p) continue;                                   // does not fit the node tables
             if (strassen_plan_set_workspace(p, req->workspace, req->workspace_bytes) != STRASSEN_OK) {
                 strassen_plan_destroy(p);
                 continue;
@@ -87,7 +165,7 @@ extern "C" int strassen_autotune(const strassen_tune_request *req, strassen_tune
             ++tried;
             strassen_tune_entry ent;
             memset(&ent, 0, sizeof ent);
-            ent.cutoff = cutoff; ent.levels = int(L); ent.ms = ms_best;
+            ent.cutoff = cutoff; ent.levels = int(L); ent.ms = ms_best; ent.model_ms = cand.model;
             snprintf(ent.schedule, sizeof ent.schedule, "%s", sched.c_str());
             if (log && log_count && *log_count < log_capacity) log[(*log_count)++] = ent;
             if (best->ms < 0 || ms_best < best->ms) *best = ent;

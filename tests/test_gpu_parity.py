@@ -398,6 +398,8 @@ def test_autotune_returns_a_valid_fastest_candidate():
     assert len(log) == 1 + 2 + 4 + 8                       # L = 0..3, every B/D string
     assert {e["levels"] for e in log} == {0, 1, 2, 3}
     assert best["ms"] == min(e["ms"] for e in log) and best["ms"] > 0
+    models = [e["model_ms"] for e in log]
+    assert models == sorted(models) and models[0] > 0       # tried in the order of the cost model
     assert len(best["schedule"]) == best["levels"] and set(best["schedule"]) <= set("BD")
     # the tuned pair recreates a plan, and C holds that plan's (correct) product
     plan = Plan(n, best["cutoff"], best["schedule"])
