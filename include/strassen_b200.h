@@ -69,7 +69,7 @@ typedef enum strassen_kernel_kind {
 /* Extended plan description.  Zero-initialise, then set what differs from the default. */
 typedef struct strassen_options {
     int64_t n;              /* matrix size, >= 1                                                   */
-    int64_t cutoff;         /* recurse while the current size is > cutoff; >= 1                    */
+    int64_t cutoff;         /* recurse while the current size is > cutoff; >= 1, or 0 = chosen by the library */
     const char *schedule;   /* one 'B' or 'D' per level, top level first; NULL or "auto" = LM rule */
     int64_t batch;          /* independent products per call; 0 means 1                            */
     int64_t lda, ldb, ldc;  /* leading dimensions in elements; 0 means n                           */
@@ -120,7 +120,12 @@ typedef struct strassen_options {
  *   n        matrix size (>= 1), contiguous rows (ld = n), one product per call.
  *   cutoff   base-case size n0 (>= 1): a node of size m is split while m > cutoff, so the
  *            level sizes are m_0 = n, m_{i+1} = floor(m_i / 2); n <= cutoff gives zero
- *            levels, i.e. one classical product [Section 5.4].
+ *            levels, i.e. one classical product [Section 5.4].  0 leaves the number of steps
+ *            to the library: with an explicit schedule string it is the string's length; with
+ *            NULL / "auto" the steps (base size >= 256) and the interleaving of least estimated
+ *            time among all that fit the workspace budget are taken, by the cost model that also
+ *            orders strassen_autotune's search [Section 5.4 tunes both by measurement; that is
+ *            strassen_autotune].
  *   schedule host string, one character per level from the top: 'B' = BFS step, 'D' = DFS
  *            step [Section 3.1].  NULL or "auto" applies the Limited-Memory rule
  *            [Section 3.4] against the free memory of the current device.

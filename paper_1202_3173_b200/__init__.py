@@ -18,9 +18,11 @@ class Plan:
 
     ``schedule`` is one 'B' (breadth-first step) or 'D' (depth-first step) per recursion
     level, or None / "auto" for the Limited-Memory rule against ``workspace_budget_bytes``.
+    ``cutoff`` 0 lets the library choose the number of steps (and, with schedule None, the
+    interleaving) by its cost model.
     """
 
-    def __init__(self, n, cutoff, schedule=None, batch=1, workspace_budget_bytes=0, lda=0, ldb=0, ldc=0,
+    def __init__(self, n, cutoff=0, schedule=None, batch=1, workspace_budget_bytes=0, lda=0, ldb=0, ldc=0,
                  stride_a=0, stride_b=0, stride_c=0, flags=0):
         self.n, self.cutoff, self.batch = int(n), int(cutoff), int(batch)
         self._h = binding.strassen_plan_create_ex(n, cutoff, schedule, batch, lda, ldb, ldc, stride_a, stride_b,
@@ -118,7 +120,7 @@ class Plan:
             pass
 
 
-def matmul(A, B, cutoff=512, schedule=None, workspace_budget_bytes=0):
+def matmul(A, B, cutoff=0, schedule=None, workspace_budget_bytes=0):
     """One-shot C = A @ B for square CUDA float64 tensors (2-D, or 3-D for a batch)."""
     import torch
     batch = 1 if A.dim() == 2 else A.shape[0]

@@ -232,8 +232,8 @@ strassen_plan *create(const strassen_options &o)
     g_error.clear();
     const int64_t n = o.n, cutoff = o.cutoff;
     const int64_t batch = o.batch == 0 ? 1 : o.batch;
-    if (n < 1 || cutoff < 1 || batch < 1) {
-        fail(STRASSEN_INVALID_ARG, "n, cutoff and batch must be positive");
+    if (n < 1 || cutoff < 0 || batch < 1) {
+        fail(STRASSEN_INVALID_ARG, "n and batch must be positive, cutoff non-negative");
         return nullptr;
     }
     if (n > (int64_t(1) << 30)) {
@@ -267,24 +267,47 @@ strassen_plan *create(const strassen_options &o)
     p->host_pipeline = (o.flags & STRASSEN_FLAG_HOST_PIPELINE) != 0;
     d.scale_inside = (o.flags & STRASSEN_FLAG_SCALE_INSIDE) != 0;
     d.scale_outside = (o.flags & STRASSEN_FLAG_SCALE_OUTSIDE) != 0;
-    d.sizes = level_sizes(n, cutoff);
-    const size_t L = d.sizes.size() - 1;
     const bool want_auto = !o.schedule || strcmp(o.schedule, "auto") == 0;
-    if (want_auto) {
-        size_t budget = o.workspace_budget_bytes;
-        if (budget == 0 && L > 0) {
-            size_t free_b = 0, total_b = 0;
-            cudaError_t e = cudaMemGetInfo(&free_b, &total_b);
-            if (e != cudaSuccess) {
-                cudaGetLastError();
-                fail(STRASSEN_CUDA_ERROR, std::string("schedule \"auto\" without a workspace budget needs a CUDA device: ") +
-                                              cudaGetErrorString(e));
-                delete p;
-                return nullptr;
-            }
-            const size_t margin = size_t(1) << 30;
-            budget = free_b > margin ? free_b - margin : 0;
+    size_t budget = o.workspace_budget_bytes;
+    if (want_auto && budget == 0 && (cutoff == 0 || n > cutoff)) {
+        size_t free_b = 0, total_b = 0;
+        cudaError_t e = cudaMemGetInfo(&free_b, &total_b);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            fail(STRASSEN_CUDA_ERROR, std::string("schedule \"auto\" without a workspace budget needs a CUDA device: ") +
+                                          cudaGetErrorString(e));
+            delete p;
+            return nullptr;
         }
+        const size_t margin = size_t(1) << 30;
+        budget = free_b > margin ? free_b - margin : 0;
+    }
+    if (cutoff == 0 && want_auto) {
+        // number of steps and interleaving by the cost model, among everything that fits the budget; bases
+        // below 256 are left out: there the passes are latency-bound and the model, built on rates, is too kind
+        if (!model_choice(n, batch, int64_t(budget / 8), 256, &d.sizes, &d.schedule)) {
+            fail(STRASSEN_WORKSPACE_TOO_SMALL, "no plan fits the workspace budget");
+            delete p;
+            return nullptr;
+        }
+    } else if (cutoff == 0) {
+        // the schedule string fixes the number of steps
+        const size_t steps = strlen(o.schedule);
+        d.sizes.assign(1, n);
+        while (d.sizes.size() <= steps && d.sizes.back() >= 2) d.sizes.push_back(d.sizes.back() / 2);
+        if (d.sizes.size() != steps + 1) {
+            fail(STRASSEN_BAD_SCHEDULE, "the schedule has more steps than n can be halved");
+            delete p;
+            return nullptr;
+        }
+    } else {
+        d.sizes = level_sizes(n, cutoff);
+    }
+    d.cutoff = d.sizes.back();
+    const size_t L = d.sizes.size() - 1;
+    if (cutoff == 0 && want_auto) {
+        // schedule chosen above
+    } else if (want_auto) {
         if (!lm_schedule(d.sizes, batch, int64_t(budget / 8), &d.schedule)) {
             fail(STRASSEN_WORKSPACE_TOO_SMALL, "even the all-DFS schedule does not fit the workspace budget");
             delete p;

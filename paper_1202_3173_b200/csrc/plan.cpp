@@ -2,6 +2,8 @@
 // (Limited-Memory rule, Section 3.4), workspace carve-up, node tables and the launch list.
 #include "plan.h"
 
+#include "kernels.h"
+
 #include <limits>
 
 namespace strassen {
@@ -195,6 +197,92 @@ int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched
     while (level + run < L && sched[level + run] == 'B' && (run == 0 || (sizes[level + run] & 1) == 0)) ++run;
     if (run <= 1) return 1;
     return run % max_fused == 0 ? max_fused : run % max_fused;
+}
+
+// Estimate of one product's time from the quantities the kernels are bound by (measured on B200): the base
+// products at the DMMA rate of their tiling, everything else as HBM bytes, a few microseconds per launch.
+// Only used to decide which candidates are tried first; the choice itself is by measurement.
+double plan_model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch)
+{
+    const int L = int(sched.size());
+    const double hbm = 6.2e12, launch_us = 3.0;
+    double bytes = 0.0, launches = 0.0, visits = double(batch), sequential = 1.0;   // node visits at the current level
+    for (int level = 0; level < L;) {
+        const double m = double(sizes[level]), h = double(sizes[level + 1]);
+        if (sizes[level] & 1) {
+            bytes += visits * 2.0 * m * m * 8.0;      // last column and last row: each reads one operand in full
+            launches += 2.0 * sequential;
+        }
+        if (sched[level] == 'D') {
+            bytes += visits * 57.0 * h * h * 8.0;     // 30 h^2 to form the operands one at a time, 27 h^2 to fold the products
+            launches += 12.0 * sequential;
+            visits *= 7.0;
+            sequential *= 7.0;
+            ++level;
+            continue;
+        }
+        const int g = fused_group_size(sizes, sched, level, 3);
+        const double words = g == 1 ? 27.0 : g == 2 ? 28.0 + 16.25 : 49.0 + 25.5;    // per parent, in h^2 of its children
+        bytes += visits * words * h * h * 8.0;
+        launches += 2.0 * sequential;
+        for (int i = 0; i < g; ++i) visits *= 7.0;
+        level += g;
+    }
+    const int64_t b = sizes[L];
+    const double leaves = visits, kp = double((b + 15) / 16 * 16);
+    const int rem = gemm_thin_remainder(b);
+    double us = 0.0;
+    if (b - rem > 0) {
+        GemmRegion regions[4];
+        const int64_t count = leaves > 4.0e9 ? int64_t(4e9) : int64_t(leaves);
+        const int nreg = gemm_regions(b - rem, count, kNominalSMs, regions);
+        const double wide_tile_us = kp / 16.0 * 2.147 + 1.1;      // one 128 x 128 tile on an SM: per 16-deep slab and per tile
+        for (int i = 0; i < nreg; ++i) {
+            const GemmRegion &r = regions[i];
+            const int t = r.small ? 64 : 128;
+            const double tiles = double((r.row_end - r.row0 + t - 1) / t) * double((r.col_end - r.col0 + t - 1) / t) * double(r.leaves);
+            const double slots = r.small ? 2.0 * kNominalSMs : double(kNominalSMs);
+            const double tile_us = r.small ? wide_tile_us * 0.5 / 0.88 : wide_tile_us;
+            double rounds = tiles / sequential / slots;          // per launch: a DFS level above runs its sub-trees one by one
+            if (rounds < 1.0) rounds = 1.0;
+            us += rounds * tile_us * sequential;
+            launches += sequential;
+        }
+    }
+    if (rem) {
+        bytes += leaves * 2.0 * double(b) * double(b) * 8.0;
+        launches += 2.0 * sequential;
+    }
+    return us * 1e-3 + bytes / hbm * 1e3 + launches * launch_us * 1e-3;
+}
+
+
+bool model_choice(int64_t n, int64_t batch, int64_t budget_words, int64_t min_base, std::vector<int64_t> *sizes_out,
+                  std::string *sched_out)
+{
+    std::vector<int64_t> chain{n};
+    while (chain.back() / 2 >= min_base && chain.size() <= 10) chain.push_back(chain.back() / 2);
+    double best = -1.0;
+    for (size_t L = 0; L < chain.size(); ++L) {
+        const std::vector<int64_t> sizes(chain.begin(), chain.begin() + L + 1);
+        for (unsigned mask = 0; mask < (1u << L); ++mask) {
+            std::string sched(L, 'B');
+            for (size_t i = 0; i < L; ++i)
+                if (mask >> i & 1) sched[i] = 'D';
+            const int64_t words = actual_workspace_words(sizes, sched, batch);
+            if (words < 0 || words > budget_words) continue;
+            double nodes = double(batch), level_nodes = double(batch);      // entries the node tables would need
+            for (size_t i = 0; i < L; ++i) nodes += (level_nodes *= 7.0);
+            if (nodes > double(kMaxNodes)) continue;
+            const double ms = plan_model_ms(sizes, sched, batch);
+            if (best < 0 || ms < best) {
+                best = ms;
+                *sizes_out = sizes;
+                *sched_out = sched;
+            }
+        }
+    }
+    return best >= 0;
 }
 
 std::vector<int64_t> level_sizes(int64_t n, int64_t cutoff)

@@ -106,6 +106,16 @@ struct PlanDesc {
 // `sched` with level sizes `sizes`; 1 for a DFS level.
 int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused);
 
+// Cost-model estimate (milliseconds on a B200) of one product with level sizes `sizes` (m_0 .. m_L) and
+// schedule `sched`; orders the autotuner's search and picks plans created with cutoff 0.
+double plan_model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch);
+
+// The (level sizes, schedule) of least estimated time among all step counts whose base size is >= min_base
+// and all B/D strings whose workspace fits budget_words.  False if nothing fits (cannot happen: zero levels
+// need no workspace).
+bool model_choice(int64_t n, int64_t batch, int64_t budget_words, int64_t min_base, std::vector<int64_t> *sizes_out,
+                  std::string *sched_out);
+
 // Level sizes m_0 = n, m_{i+1} = floor(m_i / 2) while m_i > cutoff.
 std::vector<int64_t> level_sizes(int64_t n, int64_t cutoff);
 

@@ -26,63 +26,6 @@ int tune_fail(int status, const std::string &msg)
     return status;
 }
 
-// Estimate of one product's time from the quantities the kernels are bound by (measured on B200): the base
-// products at the DMMA rate of their tiling, everything else as HBM bytes, a few microseconds per launch.
-// Only used to decide which candidates are tried first; the choice itself is by measurement.
-double model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch)
-{
-    const int L = int(sched.size());
-    const double hbm = 6.2e12, launch_us = 3.0;
-    double bytes = 0.0, launches = 0.0, visits = double(batch), sequential = 1.0;   // node visits at the current level
-    for (int level = 0; level < L;) {
-        const double m = double(sizes[level]), h = double(sizes[level + 1]);
-        if (sizes[level] & 1) {
-            bytes += visits * 2.0 * m * m * 8.0;      // last column and last row: each reads one operand in full
-            launches += 2.0 * sequential;
-        }
-        if (sched[level] == 'D') {
-            bytes += visits * 57.0 * h * h * 8.0;     // 30 h^2 to form the operands one at a time, 27 h^2 to fold the products
-            launches += 12.0 * sequential;
-            visits *= 7.0;
-            sequential *= 7.0;
-            ++level;
-            continue;
-        }
-        const int g = fused_group_size(sizes, sched, level, 3);
-        const double words = g == 1 ? 27.0 : g == 2 ? 28.0 + 16.25 : 49.0 + 25.5;    // per parent, in h^2 of its children
-        bytes += visits * words * h * h * 8.0;
-        launches += 2.0 * sequential;
-        for (int i = 0; i < g; ++i) visits *= 7.0;
-        level += g;
-    }
-    const int64_t b = sizes[L];
-    const double leaves = visits, kp = double((b + 15) / 16 * 16);
-    const int rem = gemm_thin_remainder(b);
-    double us = 0.0;
-    if (b - rem > 0) {
-        GemmRegion regions[4];
-        const int64_t count = leaves > 4.0e9 ? int64_t(4e9) : int64_t(leaves);
-        const int nreg = gemm_regions(b - rem, count, kNominalSMs, regions);
-        const double wide_tile_us = kp / 16.0 * 2.147 + 1.1;      // one 128 x 128 tile on an SM: per 16-deep slab and per tile
-        for (int i = 0; i < nreg; ++i) {
-            const GemmRegion &r = regions[i];
-            const int t = r.small ? 64 : 128;
-            const double tiles = double((r.row_end - r.row0 + t - 1) / t) * double((r.col_end - r.col0 + t - 1) / t) * double(r.leaves);
-            const double slots = r.small ? 2.0 * kNominalSMs : double(kNominalSMs);
-            const double tile_us = r.small ? wide_tile_us * 0.5 / 0.88 : wide_tile_us;
-            double rounds = tiles / sequential / slots;          // per launch: a DFS level above runs its sub-trees one by one
-            if (rounds < 1.0) rounds = 1.0;
-            us += rounds * tile_us * sequential;
-            launches += sequential;
-        }
-    }
-    if (rem) {
-        bytes += leaves * 2.0 * double(b) * double(b) * 8.0;
-        launches += 2.0 * sequential;
-    }
-    return us * 1e-3 + bytes / hbm * 1e3 + launches * launch_us * 1e-3;
-}
-
 }  // namespace
 
 extern "C" int strassen_autotune(const strassen_tune_request *req, strassen_tune_entry *best, strassen_tune_entry *log,
@@ -126,7 +69,7 @@ extern "C" int strassen_autotune(const strassen_tune_request *req, strassen_tune
                 if (mask >> i & 1) sched[i] = 'D';
             const int64_t words = actual_workspace_words(chain, sched, batch);
             if (words < 0 || size_t(words) > req->workspace_bytes / 8) continue;       // does not fit the workspace
-            candidates.push_back(Candidate{sizes[L], sched, model_ms(chain, sched, batch)});
+            candidates.push_back(Candidate{sizes[L], sched, plan_model_ms(chain, sched, batch)});
         }
     }
     // most promising first, so that a search cut short by max_seconds has seen the likely winners

@@ -287,6 +287,18 @@ def test_item_lists_longer_than_one_launch_covers(n, cutoff, sched, flags):
     assert np.array_equal(C.cpu().numpy(), oracle.classical(A.cpu().numpy(), B.cpu().numpy()))
 
 
+@pytest.mark.parametrize("n", [700, 1500, 3001])
+def test_library_chosen_plan_gives_the_product(n):
+    # cutoff 0, schedule None: steps and interleaving picked by the cost model against the free device memory
+    from paper_1202_3173_b200 import matmul
+    A, B = inputs.pair(n, "int8", 2900 + n, device="cuda")
+    C = matmul(A, B)
+    x = torch.randint(0, 3, (n, 1), device="cuda", generator=torch.Generator("cuda").manual_seed(n)).double()
+    assert torch.equal(C @ x, A @ (B @ x))              # Freivalds, exact on small integers
+    if n <= 1500:
+        assert np.array_equal(C.cpu().numpy(), oracle.classical(A.cpu().numpy(), B.cpu().numpy()))
+
+
 def test_first_call_on_a_side_stream_sees_its_node_tables():
     # 137 257 nodes (6.6 MB of tables) uploaded by the first call, which is made on a non-blocking stream while
     # another stream keeps the host-to-device copy engine busy: the product must wait for its own tables

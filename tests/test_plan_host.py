@@ -30,7 +30,7 @@ def test_schedule_errors():
     with pytest.raises(StrassenError):
         Plan(0, 512, "")
     with pytest.raises(StrassenError):
-        Plan(64, 0, "")
+        Plan(64, -1, "")
     with pytest.raises(StrassenError):
         Plan(64, 8, "BBB", lda=32)
     with pytest.raises(StrassenError):
@@ -133,6 +133,33 @@ def test_auto_without_budget_or_device_fails_loudly():
     with pytest.raises(StrassenError) as e:
         Plan(4096, 512, "auto")
     assert "CUDA" in str(e.value)
+
+
+def test_cutoff_zero_lets_the_cost_model_choose():
+    GBb = int(1e9)
+    # the choices the measurements on a B200 confirmed (autotune finds the same plans)
+    for n, batch, budget, sched, base in [(4096, 1, 40, "BBB", 512), (16384, 1, 40, "DBBBB", 512), (12345, 1, 40, "BBB", 1543),
+                                          (47040, 1, 125, "DDBBB", 1470), (2048, 32, 40, "BBB", 256), (512, 1, 1, "B", 256),
+                                          (1000, 1, 1, "", 1000), (300, 1, 1, "", 300)]:
+        p = Plan(n, 0, None, batch=batch, workspace_budget_bytes=budget * GBb)
+        assert (p.schedule, p.base_size) == (sched, base), (n, p.schedule, p.base_size)
+        assert p.workspace_bytes <= budget * GBb
+        p.close()
+    # a tighter budget trades BFS steps for DFS steps or a larger base; nothing that does not fit is chosen
+    p = Plan(16384, 0, None, workspace_budget_bytes=2 * GBb)
+    assert p.workspace_bytes <= 2 * GBb and p.levels >= 1
+    p.close()
+    p = Plan(4096, 0, None, workspace_budget_bytes=1)       # no room at all: the classical product
+    assert p.levels == 0
+    p.close()
+    # an explicit schedule with cutoff 0 fixes the number of steps by its length
+    p = Plan(4096, 0, "BD")
+    assert p.level_sizes == [4096, 2048, 1024] and p.schedule == "BD"
+    p.close()
+    with pytest.raises(StrassenError):
+        Plan(8, 0, "BBBB")
+    with pytest.raises(StrassenError):
+        Plan(4096, -1, "B")
 
 
 def test_launch_lists():
