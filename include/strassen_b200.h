@@ -279,7 +279,7 @@ int strassen_probe_fp64(int kind, int64_t iters, void *stream, double *tflops_ou
  * cutoff floor(n / 2); the results are identical to that call's.
  *
  * Where the temporaries live: the eight operand sums, the seven products and a small node
- * table are kept in a static device array compiled into the library (about 7.9 MB, sized for
+ * table (8 entries: the product and its seven sub-products) are kept in a static device array compiled into the library (about 7.9 MB, sized for
  * n = STRASSEN_STATIC_MAX_N).  Every GPU that loads the library holds that array until the
  * process exits.  A larger n is rejected with STRASSEN_WORKSPACE_TOO_SMALL and a message that
  * names the limit; nothing is launched in that case.
@@ -291,8 +291,10 @@ int strassen_probe_fp64(int kind, int64_t iters, void *stream, double *tflops_ou
  *
  * Rules that follow from the shared array:
  *   - The first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress, with that device current) and the SM count; make that first call
- *     before starting any stream capture on that device.  Later calls do no set-up.
+ *     (cudaGetSymbolAddress, with that device current) and the SM count, and sets the
+ *     shared-memory attribute of the product kernels (cudaFuncSetAttribute) unless a plan has
+ *     done so on that device already; make that first call before starting any stream capture
+ *     on that device.  Later calls do no set-up.
  *   - All calls on a device use the same array, and it keeps whatever the previous call left
  *     in it.  No part of it needs to start at zero: every temporary is written in full before
  *     it is read.  Two calls whose kernels can overlap on the GPU (different streams without

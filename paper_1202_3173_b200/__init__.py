@@ -28,6 +28,7 @@ class Plan:
         self._h = binding.strassen_plan_create_ex(n, cutoff, schedule, batch, lda, ldb, ldc, stride_a, stride_b,
                                                   stride_c, workspace_budget_bytes, flags)
         self._ws = None
+        self._packed = not (lda or ldb or ldc or stride_a or stride_b or stride_c)
 
     # -- introspection -------------------------------------------------------------
     @property
@@ -78,15 +79,35 @@ class Plan:
             self._ws = torch.empty(need, dtype=torch.uint8, device=device)
             binding.strassen_plan_set_workspace(self._h, self._ws.data_ptr(), need)
 
-    def __call__(self, A, B, out=None):
-        """C = A @ B for CUDA float64 tensors, enqueued on the current stream."""
+    def _check(self, what, cuda, *tensors):
+        """The kernels index the tensors by the plan's n and batch alone: anything smaller than that would be
+        read or written out of bounds on the device, so shapes are checked here and not left to the library."""
         import torch
-        if not (A.is_cuda and B.is_cuda and A.dtype == torch.float64 and B.dtype == torch.float64):
-            raise ValueError("A and B must be CUDA float64 tensors (there is no CPU path)")
-        if not (A.is_contiguous() and B.is_contiguous()):
-            raise ValueError("A and B must be contiguous")
+        if not self._h:
+            raise ValueError("the plan has been closed")
+        if not self._packed:
+            raise ValueError("plans with leading dimensions or strides take raw pointers (binding.strassen_dgemm)")
+        want = (self.n, self.n) if self.batch == 1 else (self.batch, self.n, self.n)
+        for name, t in zip(what, tensors):
+            if t.dtype != torch.float64:
+                raise ValueError("%s must be float64, not %s" % (name, t.dtype))
+            if tuple(t.shape) != want and not (self.batch == 1 and tuple(t.shape) == (1,) + want):
+                raise ValueError("%s has shape %s; the plan is for %s" % (name, tuple(t.shape), want))
+            if not t.is_contiguous():
+                raise ValueError("%s must be contiguous" % name)
+            if t.is_cuda != cuda:
+                raise ValueError("%s must be a %s tensor" % (name, "CUDA" if cuda else "host"))
+            if cuda and t.device != tensors[0].device:
+                raise ValueError("%s is on %s, A on %s" % (name, t.device, tensors[0].device))
+
+    def __call__(self, A, B, out=None):
+        """C = A @ B for CUDA float64 tensors of the plan's shape, enqueued on the current stream."""
+        import torch
         if out is None:
+            self._check("AB", True, A, B)
             out = torch.empty_like(A)
+        else:
+            self._check(("A", "B", "out"), True, A, B, out)
         self._ensure_workspace(A.device)
         with torch.cuda.device(A.device):
             stream = torch.cuda.current_stream().cuda_stream
@@ -96,6 +117,7 @@ class Plan:
     def run_host(self, A, B, out):
         """The same product for host (ideally pinned) tensors, copies included, on the current stream."""
         import torch
+        self._check(("A", "B", "out"), False, A, B, out)
         self._ensure_workspace(torch.device("cuda", torch.cuda.current_device()))
         stream = torch.cuda.current_stream().cuda_stream
         binding.strassen_dgemm_host(self._h, A.data_ptr(), B.data_ptr(), out.data_ptr(), stream)
@@ -108,7 +130,12 @@ class Plan:
         return binding.strassen_plan_get_timings(self._h)
 
     def close(self):
+        """Destroy the plan.  Launches that still use its workspace may be in flight on any stream, so the device
+        the workspace lives on is synchronised before the memory goes back to torch's allocator."""
         if self._h:
+            if self._ws is not None:
+                import torch
+                torch.cuda.synchronize(self._ws.device)
             binding.strassen_plan_destroy(self._h)
             self._h = None
             self._ws = None
@@ -123,6 +150,9 @@ class Plan:
 def matmul(A, B, cutoff=0, schedule=None, workspace_budget_bytes=0):
     """One-shot C = A @ B for square CUDA float64 tensors (2-D, or 3-D for a batch)."""
     import torch
+    if A.dim() not in (2, 3) or A.shape != B.shape or A.shape[-1] != A.shape[-2]:
+        raise ValueError("A and B must be square matrices (or batches of them) of equal shape, got %s and %s"
+                         % (tuple(A.shape), tuple(B.shape)))
     batch = 1 if A.dim() == 2 else A.shape[0]
     n = A.shape[-1]
     plan = Plan(n, cutoff, schedule, batch=batch, workspace_budget_bytes=workspace_budget_bytes)
@@ -140,6 +170,9 @@ def autotune(A, B, workspace_budget_bytes, min_base=0, repetitions=0, max_second
     computed with the winning plan.  torch supplies C and the workspace; the search itself runs
     inside the library (strassen_autotune)."""
     import torch
+    if (A.dim() not in (2, 3) or A.shape != B.shape or A.shape[-1] != A.shape[-2] or not (A.is_cuda and B.is_cuda)
+            or A.dtype != torch.float64 or B.dtype != torch.float64 or not (A.is_contiguous() and B.is_contiguous())):
+        raise ValueError("A and B must be contiguous square CUDA float64 matrices (or batches) of equal shape")
     batch = 1 if A.dim() == 2 else A.shape[0]
     n = A.shape[-1]
     C = torch.empty_like(A)

@@ -63,9 +63,15 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 def ensure_built() -> str:
-    """Build only if the shared library is absent (used by the tests, the smoke check and the benchmark, so that a
-    checkout without build products still runs where nvcc is available)."""
-    return LIB if os.path.exists(LIB) else build()
+    """The shared library, rebuilt first if it is absent or older than any source or header (used by the tests, the
+    smoke check and the benchmark, so that what they run is what the sources say).  Where the library exists and no
+    compiler does, it is used as it is."""
+    try:
+        return build()
+    except OSError:          # no nvcc on this machine (a compile error is a RuntimeError and is not swallowed)
+        if os.path.exists(LIB):
+            return LIB
+        raise
 
 
 if __name__ == "__main__":

@@ -96,6 +96,25 @@ cudaEvent_t take_event(strassen_plan *p)
     return e;
 }
 
+// Wait for the timing events recorded so far, add their durations to the per-family sums and recycle the events.
+int harvest_timings(strassen_plan *p)
+{
+    for (TimedLaunch &t : p->pending) {
+        cudaError_t e = cudaEventSynchronize(t.stop);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, t.start, t.stop);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventElapsedTime");
+        p->acc_ms[t.kind] += double(ms);
+        p->free_events.push_back(t.start);
+        p->free_events.push_back(t.stop);
+    }
+    p->pending.clear();
+    return STRASSEN_OK;
+}
+
+constexpr size_t kMaxPendingTimings = 1 << 16;   // event pairs kept before a timed call folds them into the sums
+
 // First use on a device: node tables, SM count, workspace.
 int ensure_device_state(strassen_plan *p, cudaStream_t stream)
 {
@@ -157,6 +176,11 @@ int ensure_device_state(strassen_plan *p, cudaStream_t stream)
 int enqueue_launches(strassen_plan *p, const Bases &bases, bool bases16, cudaStream_t stream, bool timed)
 {
     int launched = 0;
+    if (timed && p->pending.size() + p->d.launches.size() > kMaxPendingTimings) {
+        // timing left on and never read: fold what has accumulated (waits for those launches) instead of growing
+        const int rc = harvest_timings(p);
+        if (rc != STRASSEN_OK) return rc;
+    }
     for (const Launch &op : p->d.launches) {
         const bool vec = op.vec_ok && bases16;
         TimedLaunch t{family(op.kind), nullptr, nullptr};
@@ -388,6 +412,11 @@ int strassen_dgemm(strassen_plan *p, const double *A, const double *B, double *C
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const int rc = ensure_device_state(p, stream);
     if (rc != STRASSEN_OK) return rc;
+    if (p->ws && d.ws_words > 0) {
+        const int64_t ww = d.ws_words;
+        if (overlap(p->ws, ww, A, wa) || overlap(p->ws, ww, B, wb) || overlap(p->ws, ww, C, wc))
+            return fail(STRASSEN_ALIAS, "the workspace overlaps A, B or C");
+    }
     Bases bases;
     bases.p[BASE_A] = const_cast<double *>(A);
     bases.p[BASE_B] = const_cast<double *>(B);
@@ -583,17 +612,8 @@ int strassen_plan_get_timings(strassen_plan *p, double *ms_out)
 {
     g_error.clear();
     if (!p || !ms_out) return fail(STRASSEN_INVALID_ARG, "plan and output must be non-NULL");
-    for (TimedLaunch &t : p->pending) {
-        cudaError_t e = cudaEventSynchronize(t.stop);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
-        float ms = 0.f;
-        e = cudaEventElapsedTime(&ms, t.start, t.stop);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaEventElapsedTime");
-        p->acc_ms[t.kind] += double(ms);
-        p->free_events.push_back(t.start);
-        p->free_events.push_back(t.stop);
-    }
-    p->pending.clear();
+    const int rc = harvest_timings(p);
+    if (rc != STRASSEN_OK) return rc;
     for (int k = 0; k < STRASSEN_K_COUNT; ++k) {
         ms_out[k] = p->acc_ms[k];
         p->acc_ms[k] = 0.0;

@@ -24,6 +24,8 @@
 //     with an odd leading dimension) use 8-byte copies.
 #include "kernels.h"
 
+#include <atomic>
+
 namespace strassen {
 
 namespace {
@@ -363,7 +365,9 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, GemmRegion reg, int
 
 namespace {
 
-bool g_configured[64];   // per device: kernels opted in to > 48 KB of dynamic shared memory
+// Per device: kernels opted in to > 48 KB of dynamic shared memory.  Atomic because two host threads may make
+// their first call at once; the set-up itself is idempotent, so both may run it.
+std::atomic<bool> g_configured[64];
 
 }  // namespace
 
@@ -377,7 +381,7 @@ cudaError_t launch_cfg(const Node *nodes, const Bases &bases, const GemmRegion &
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !g_configured[dev]) {
+    if (dev < 0 || dev >= 64 || !g_configured[dev].load(std::memory_order_acquire)) {
         e = configure_gemm_kernels();
         if (e != cudaSuccess) return e;
     }
@@ -398,12 +402,12 @@ cudaError_t configure_gemm_kernels()
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64 && g_configured[dev]) return cudaSuccess;
+    if (dev >= 0 && dev < 64 && g_configured[dev].load(std::memory_order_acquire)) return cudaSuccess;
     e = cudaFuncSetAttribute(gemm_f64_kernel<CfgWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgWide::SMEM_BYTES));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(gemm_f64_kernel<CfgSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgSmall::SMEM_BYTES));
     if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) g_configured[dev] = true;
+    if (dev >= 0 && dev < 64) g_configured[dev].store(true, std::memory_order_release);
     return cudaSuccess;
 }
 

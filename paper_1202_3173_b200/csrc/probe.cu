@@ -9,7 +9,12 @@ namespace {
 constexpr int PROBE_THREADS = 256;
 constexpr int CHAINS = 8;
 
-__global__ void __launch_bounds__(PROBE_THREADS) probe_dfma_kernel(double *out, long long iters, double x, double y)
+// Keeps the loops alive without an output buffer (so the probe allocates nothing): a thread stores its sum only
+// if it equals a value the loops cannot produce.
+__device__ double g_probe_sink;
+constexpr double kNever = -1.2345678901234567e300;
+
+__global__ void __launch_bounds__(PROBE_THREADS) probe_dfma_kernel(long long iters, double x, double y)
 {
     double a[CHAINS];
 #pragma unroll
@@ -21,11 +26,11 @@ __global__ void __launch_bounds__(PROBE_THREADS) probe_dfma_kernel(double *out, 
     double s = 0.0;
 #pragma unroll
     for (int c = 0; c < CHAINS; ++c) s += a[c];
-    out[blockIdx.x * PROBE_THREADS + threadIdx.x] = s;
+    if (s == kNever) g_probe_sink = s;
 }
 
 template <int KIND>
-__global__ void __launch_bounds__(PROBE_THREADS) probe_dmma_kernel(double *out, long long iters, double x, double y)
+__global__ void __launch_bounds__(PROBE_THREADS) probe_dmma_kernel(long long iters, double x, double y)
 {
     double d[CHAINS][4];
 #pragma unroll
@@ -57,7 +62,7 @@ __global__ void __launch_bounds__(PROBE_THREADS) probe_dmma_kernel(double *out, 
     double s = 0.0;
 #pragma unroll
     for (int c = 0; c < CHAINS; ++c) s += d[c][0] + d[c][1] + d[c][2] + d[c][3];
-    out[blockIdx.x * PROBE_THREADS + threadIdx.x] = s;
+    if (s == kNever) g_probe_sink = s;
 }
 
 }  // namespace
@@ -71,9 +76,6 @@ cudaError_t probe_fp64(int kind, long long iters, cudaStream_t stream, double *t
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     const int blocks = sms * 4;
-    double *out = nullptr;
-    e = cudaMalloc(&out, size_t(blocks) * PROBE_THREADS * sizeof(double));
-    if (e != cudaSuccess) return e;
     cudaEvent_t t0, t1;
     cudaEventCreate(&t0);
     cudaEventCreate(&t1);
@@ -81,11 +83,11 @@ cudaError_t probe_fp64(int kind, long long iters, cudaStream_t stream, double *t
     for (int rep = 0; rep < 2; ++rep) {   // first pass warms up, second is timed
         cudaEventRecord(t0, stream);
         switch (kind) {
-        case 0: probe_dfma_kernel<<<blocks, PROBE_THREADS, 0, stream>>>(out, iters, 0.999999, 1e-9); break;
-        case 1: probe_dmma_kernel<1><<<blocks, PROBE_THREADS, 0, stream>>>(out, iters, 1e-3, 1e-3); break;
-        case 2: probe_dmma_kernel<2><<<blocks, PROBE_THREADS, 0, stream>>>(out, iters, 1e-3, 1e-3); break;
-        case 3: probe_dmma_kernel<3><<<blocks, PROBE_THREADS, 0, stream>>>(out, iters, 1e-3, 1e-3); break;
-        default: probe_dmma_kernel<4><<<blocks, PROBE_THREADS, 0, stream>>>(out, iters, 1e-3, 1e-3); break;
+        case 0: probe_dfma_kernel<<<blocks, PROBE_THREADS, 0, stream>>>(iters, 0.999999, 1e-9); break;
+        case 1: probe_dmma_kernel<1><<<blocks, PROBE_THREADS, 0, stream>>>(iters, 1e-3, 1e-3); break;
+        case 2: probe_dmma_kernel<2><<<blocks, PROBE_THREADS, 0, stream>>>(iters, 1e-3, 1e-3); break;
+        case 3: probe_dmma_kernel<3><<<blocks, PROBE_THREADS, 0, stream>>>(iters, 1e-3, 1e-3); break;
+        default: probe_dmma_kernel<4><<<blocks, PROBE_THREADS, 0, stream>>>(iters, 1e-3, 1e-3); break;
         }
         cudaEventRecord(t1, stream);
         e = cudaEventSynchronize(t1);
@@ -94,7 +96,6 @@ cudaError_t probe_fp64(int kind, long long iters, cudaStream_t stream, double *t
     }
     cudaEventDestroy(t0);
     cudaEventDestroy(t1);
-    cudaFree(out);
     if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

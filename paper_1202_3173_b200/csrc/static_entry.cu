@@ -3,6 +3,7 @@
 // kernels index) live in a file-scope device array instead of a cudaMalloc'd workspace.
 #include "strassen_b200.h"
 
+#include <atomic>
 #include <string>
 
 #include "kernels.h"
@@ -14,7 +15,7 @@ namespace {
 
 constexpr int64_t kMaxN = STRASSEN_STATIC_MAX_N;
 constexpr int64_t kMaxH = kMaxN / 2;
-constexpr int64_t kTableWords = 64;                         // 9 nodes of 48 bytes fit in 512 bytes
+constexpr int64_t kTableWords = 64;                         // 8 nodes of 48 bytes (384 of the 512 bytes reserved)
 constexpr int64_t kMatWords = kMaxH * kMaxH;                // one quarter-size matrix at the largest n
 constexpr int64_t kScratchWords = kTableWords + 15 * kMatWords;
 
@@ -23,8 +24,10 @@ constexpr int64_t kScratchWords = kTableWords + 15 * kMatWords;
 static __device__ __align__(256) double g_static_scratch[kScratchWords];
 
 constexpr int kMaxDevices = 64;
-double *g_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device ordinal
-int g_sm_count[kMaxDevices];
+// Device address of g_static_scratch and SM count, per device ordinal.  Atomics: two host threads may make
+// their first call on a device at once; both then resolve the same values, and the pointer is published last.
+std::atomic<double *> g_scratch_ptr[kMaxDevices];
+std::atomic<int> g_sm_count[kMaxDevices];
 
 // Writes the node table of a one-level tree: entry 0 is the parent (A, B, C as given), entries
 // 1..7 its children j = 0..6 (Appendix A): quadrant operands point into A / B, operand sums
@@ -86,9 +89,10 @@ extern "C" int strassen_dgemm_static(int64_t n, const double *A, const double *B
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return static_fail(STRASSEN_CUDA_ERROR, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
     if (dev < 0 || dev >= kMaxDevices) return static_fail(STRASSEN_INVALID_ARG, "device ordinal out of range");
-    if (!g_scratch_ptr[dev]) {
+    if (!g_scratch_ptr[dev].load(std::memory_order_acquire)) {
         // First call on this device: resolve the device address of the scratch array (with this
-        // device current) and read the SM count.  Neither allocates.
+        // device current), read the SM count, opt the product kernels in to their shared memory.
+        // None of these allocates.
         double *ptr = nullptr;
         e = cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_scratch);
         if (e != cudaSuccess || !ptr)
@@ -96,10 +100,12 @@ extern "C" int strassen_dgemm_static(int64_t n, const double *A, const double *B
         int sms = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return static_fail(STRASSEN_CUDA_ERROR, std::string("cudaDeviceGetAttribute: ") + cudaGetErrorString(e));
-        g_sm_count[dev] = sms;
-        g_scratch_ptr[dev] = ptr;
+        e = configure_gemm_kernels();        // shared-memory attribute of the product kernels: no allocation either
+        if (e != cudaSuccess) return static_fail(STRASSEN_CUDA_ERROR, std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e));
+        g_sm_count[dev].store(sms, std::memory_order_relaxed);
+        g_scratch_ptr[dev].store(ptr, std::memory_order_release);
     }
-    double *scratch = g_scratch_ptr[dev];
+    double *scratch = g_scratch_ptr[dev].load(std::memory_order_acquire);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
 
     const int64_t h = n / 2;
@@ -132,7 +138,7 @@ extern "C" int strassen_dgemm_static(int64_t n, const double *A, const double *B
 
     int launched = 0;
     e = launch_form(tab, form, bases, vec, stream, &launched);
-    if (e == cudaSuccess) e = launch_gemm(tab, gemm, bases, g_sm_count[dev], stream, &launched);
+    if (e == cudaSuccess) e = launch_gemm(tab, gemm, bases, g_sm_count[dev].load(std::memory_order_relaxed), stream, &launched);
     if (e == cudaSuccess) e = launch_recombine(tab, rec, bases, vec, stream, &launched);
     if (e == cudaSuccess && (n & 1)) e = launch_peel(tab, peel, bases, stream, &launched);
     if (e != cudaSuccess) return static_fail(STRASSEN_CUDA_ERROR, std::string("kernel launch: ") + cudaGetErrorString(e));

@@ -31,13 +31,16 @@ def run_plan(n, cutoff, sched, A, B, batch=1, **kw):
     return C
 
 
-def check_full(n, cutoff, sched, dist, seed, batch=1):
-    """Whole-matrix comparison with the classical oracle."""
+def check_full(n, cutoff, sched, dist, seed, batch=1, members=None, **kw):
+    """Whole-matrix comparison with the classical oracle (for a batch: every member, or those listed)."""
     A, B = inputs.pair(n, dist, seed, device="cuda", batch=None if batch == 1 else batch)
-    C = run_plan(n, cutoff, sched, A, B, batch=batch)
-    Ah, Bh, Ch = A.cpu().numpy(), B.cpu().numpy(), C.cpu().numpy()
-    assert not np.isnan(Ch).any(), "some element of C was never written"
-    members = [(Ah, Bh, Ch)] if batch == 1 else [(Ah[b], Bh[b], Ch[b]) for b in range(batch)]
+    C = run_plan(n, cutoff, sched, A, B, batch=batch, **kw)
+    assert not bool(torch.isnan(C).any()), "some element of C was never written"
+    if batch == 1:
+        members = [(A.cpu().numpy(), B.cpu().numpy(), C.cpu().numpy())]
+    else:
+        members = [(A[b].cpu().numpy(), B[b].cpu().numpy(), C[b].cpu().numpy())
+                   for b in (range(batch) if members is None else members)]
     worst = 0.0
     for a, b, c in members:
         ref = oracle.classical(a, b)

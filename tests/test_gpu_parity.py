@@ -223,8 +223,7 @@ def test_three_level_passes_cover_odd_parents_ragged_tiles_and_stacked_groups(n,
     fused = run_plan(n, cutoff, sched, A, B)
     single = run_plan(n, cutoff, sched, A, B, flags=binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
     assert torch.equal(fused, single)
-    if n <= 1100:
-        check_full(n, cutoff, sched, dist, n + 11)
+    check_full(n, cutoff, sched, dist, n + 11)          # and the oracle's definition, whole matrix
 
 
 def test_batch_with_two_level_passes():
@@ -273,6 +272,16 @@ def test_errors_on_device():
     with pytest.raises(StrassenError) as e:
         binding.strassen_plan_set_workspace(plan.handle, small.data_ptr(), 1024)
     assert e.value.status == -3
+    # a workspace that overlaps an operand is refused before anything is launched
+    need = plan.workspace_bytes
+    big = torch.zeros(need // 8 + 64 * 64 + 64, dtype=torch.float64, device="cuda")
+    Ain = big[need // 8 - 32: need // 8 - 32 + 64 * 64].view(64, 64)        # starts inside the workspace range
+    assert big.data_ptr() % 256 == 0
+    binding.strassen_plan_set_workspace(plan.handle, big.data_ptr(), need)
+    C = torch.empty_like(B)
+    with pytest.raises(StrassenError) as e:
+        binding.strassen_dgemm(plan.handle, Ain.data_ptr(), B.data_ptr(), C.data_ptr(), 0)
+    assert e.value.status == -4 and "workspace" in str(e.value)
     plan.close()
 
 
@@ -366,6 +375,8 @@ def test_outside_scaling_meets_the_row_column_wise_bound():
     scaled = run_plan(n, cutoff, sched, A, B, flags=binding.STRASSEN_FLAG_SCALE_OUTSIDE).cpu().numpy()
     rows = A.abs().amax(dim=1).cpu().numpy()
     cols = B.abs().amax(dim=0).cpu().numpy()
+    # 4e-11 = 1e-11 (the norm-wise constant) x 2 x 2: the scaled factors have rows of A and columns of B in [1, 2),
+    # and scaling back multiplies entry (i, j) by factors that are at most max_k|A_ik| and max_k|B_kj|
     entry_bound = 4e-11 * n * rows[:, None] * cols[None, :]
     assert np.all(np.abs(scaled - ref) <= entry_bound)
     assert not np.all(np.abs(plain - ref) <= entry_bound)
@@ -424,19 +435,24 @@ def test_autotune_returns_a_valid_fastest_candidate():
     assert best0["levels"] == 0 and len(log0) == 1
 
 
-# ---- full-size configurations: sampled blocks of the definition + exact integer variant ----
+# ---- full-size configurations --------------------------------------------------------------
+# n <= 4096: the whole matrix against the classical oracle (a few seconds of host time each); larger n:
+# sampled blocks of the definition that contain every recursion boundary, exact on the integer variant,
+# plus Freivalds over the whole matrix.
 
 def test_config_n4096_bbb_full_size():
-    check_sampled(4096, 512, "BBB", "int8", 2501)
-    r = check_sampled(4096, 512, "BBB", "uniform", 2001)
+    check_full(4096, 512, "BBB", "int8", 2501)
+    r = check_full(4096, 512, "BBB", "uniform", 2001)
     assert r < 1e-2
+    check_sampled(4096, 512, "BBB", "int8", 2501)       # the sampled checker itself, where the full answer is known
 
 
 def test_config_batch32_n2048_bb_full_size():
     if _free_bytes() < 20 * GB:
         pytest.skip("needs 15 GB")
-    check_sampled(2048, 512, "BB", "int8", 5502, batch=32, members=(0, 13, 31))
-    check_sampled(2048, 512, "BB", "uniform", 5002, batch=32, members=(0, 31))
+    check_full(2048, 512, "BB", "int8", 5502, batch=32, members=(0, 13, 31))
+    check_full(2048, 512, "BB", "uniform", 5002, batch=32, members=(0, 31))
+    check_sampled(2048, 512, "BB", "int8", 5502, batch=32, members=tuple(range(1, 31, 4)))
 
 
 def test_config_n12345_peeling_full_size():

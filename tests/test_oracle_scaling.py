@@ -57,7 +57,10 @@ def test_outside_scaling_gives_the_row_column_wise_bound():
     plain, _ = oracle.strassen_winograd(A, B, 32)
     scaled, _ = oracle.scaled_strassen_winograd(A, B, 32)
     rows, cols = np.abs(A).max(axis=1), np.abs(B).max(axis=0)
-    bound = 4e-11 * n * rows[:, None] * cols[None, :]      # |C_ij - C^_ij| <= f(n) eps ||A(i,:)|| ||B(:,j)||
+    # |C_ij - C^_ij| <= f(n) eps ||A(i,:)|| ||B(:,j)||.  The constant: the scaled factors have every row of A and
+    # column of B in [1, 2), so the norm-wise bound 1e-11 n max|A'| max|B'| is below 1e-11 n 2 2 = 4e-11 n for them;
+    # scaling C back multiplies entry (i, j) by 2^-e1_i 2^-e3_j, and 2^-e1_i <= max_k|A_ik|, 2^-e3_j <= max_k|B_kj|.
+    bound = 4e-11 * n * rows[:, None] * cols[None, :]
     assert np.all(np.abs(scaled - ref) <= bound)
     assert not np.all(np.abs(plain - ref) <= bound)        # the unscaled recursion only meets the norm-wise bound
     assert np.abs(plain - ref).max() <= 1e-11 * n * np.abs(A).max() * np.abs(B).max()

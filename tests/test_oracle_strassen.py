@@ -172,5 +172,12 @@ def test_float_error_within_the_norm_wise_bound(n, cutoff, sched, dist):
 
 
 def test_effective_gflops_definition():
-    assert oracle.effective_gflops(94080, 1.0) == 2 * 94080 ** 3 / 1e9
-    assert oracle.effective_gflops(2048, 0.5, batch=32) == 32 * 2 * 2048 ** 3 / 0.5e9
+    # Section 5.2, values worked by hand: 2 * 1000^3 flop in 2 s is exactly 1 GFLOP/s; 2 * 2000^3 = 1.6e10 flop
+    # in 4 s is 4 GFLOP/s; 2 * 2048^3 = 17 179 869 184 flop, 32 of them in half a second: 1099.511627776 GFLOP/s;
+    # halving the time doubles the rate, and the rate grows with the cube of n
+    assert oracle.effective_gflops(1000, 2.0) == 1.0
+    assert oracle.effective_gflops(2000, 4.0) == 4.0
+    assert oracle.effective_gflops(2048, 0.5, batch=32) == pytest.approx(1099.511627776, rel=1e-15)
+    assert oracle.effective_gflops(94080, 1.0) == pytest.approx(1665412.890624, rel=1e-15)   # 94080^2 = 8 851 046 400; 2 * 94080^3 = 1 665 412 890 624 000
+    assert oracle.effective_gflops(500, 1.0) * 8 == oracle.effective_gflops(1000, 1.0)
+    assert oracle.effective_gflops(1000, 1.0) == 2 * oracle.effective_gflops(1000, 2.0)

@@ -242,3 +242,32 @@ def test_batch_is_extra_live_nodes():
     assert p.base_products == 32 * 49
     assert p.launches_by_kind()["gemm"] == 1
     p.close()
+
+
+def test_python_plan_checks_shapes_before_any_pointer_reaches_the_library():
+    """The kernels index their operands by the plan's n and batch only, so a smaller tensor would be read or
+    written out of bounds on the device: the Python layer must refuse it (host-only: nothing is launched)."""
+    import torch
+    from paper_1202_3173_b200 import Plan, matmul
+    plan = Plan(64, 16, "BB")
+    ok = torch.zeros((64, 64), dtype=torch.float64)
+    with pytest.raises(ValueError, match="CUDA"):
+        plan(ok, ok)                                            # host tensors on the device entry point
+    for bad in (torch.zeros((32, 64), dtype=torch.float64), torch.zeros((64, 64), dtype=torch.float32),
+                torch.zeros((64, 128), dtype=torch.float64)[:, ::2], torch.zeros((2, 64, 64), dtype=torch.float64)):
+        with pytest.raises(ValueError):
+            plan.run_host(bad, ok, ok.clone())
+        with pytest.raises(ValueError):
+            plan.run_host(ok, ok, bad)
+    batched = Plan(64, 16, "BB", batch=3)
+    with pytest.raises(ValueError, match="shape"):
+        batched.run_host(ok, ok, ok.clone())
+    strided = Plan(64, 16, "BB", lda=80)
+    with pytest.raises(ValueError, match="raw pointers"):
+        strided.run_host(ok, ok, ok.clone())
+    with pytest.raises(ValueError, match="square"):
+        matmul(torch.zeros((64, 32), dtype=torch.float64), torch.zeros((32, 64), dtype=torch.float64))
+    plan.close()
+    with pytest.raises(ValueError, match="closed"):
+        plan.run_host(ok, ok, ok.clone())
+    batched.close(); strided.close()

@@ -1,6 +1,11 @@
 """strassen_dgemm_static: the entry point for callers that may not allocate device memory
 (its temporaries sit in a static device array inside the library).  It must give the same
 result as strassen_dgemm with one level, on consecutive calls that reuse the shared array."""
+import os
+import subprocess
+import sys
+import textwrap
+
 import numpy as np
 import pytest
 import torch
@@ -20,7 +25,7 @@ def _reference_path(n, A, B):
     return C
 
 
-@pytest.mark.parametrize("n", [512, 301, 64])
+@pytest.mark.parametrize("n", [512, 511, 301, 64, 3, 2])
 def test_static_entry_matches_the_planned_entry_twice_in_a_row(n):
     stream = torch.cuda.current_stream().cuda_stream
     for call, (dist, seed) in enumerate((("uniform", 71), ("int8", 72))):
@@ -51,3 +56,25 @@ def test_static_entry_rejects_sizes_beyond_its_array():
     with pytest.raises(StrassenError) as e:
         binding.strassen_dgemm_static(64, A.data_ptr(), B.data_ptr(), A.data_ptr(), 0)
     assert e.value.status == -4
+
+
+def test_static_entry_alone_in_a_fresh_process():
+    """The caller this entry point is for never creates a plan: its first call on the device must do all
+    the set-up itself.  A child process calls nothing but strassen_dgemm_static, twice on one stream."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    child = textwrap.dedent("""
+        import numpy as np, torch
+        import oracle
+        from paper_1202_3173_b200 import binding, inputs
+        stream = torch.cuda.current_stream().cuda_stream
+        for n, dist, seed in ((384, "int8", 5), (511, "int8", 6), (2, "int8", 7)):
+            A, B = inputs.pair(n, dist, seed, device="cuda")
+            for call in range(2):
+                C = torch.full_like(A, float("nan"))
+                binding.strassen_dgemm_static(n, A.data_ptr(), B.data_ptr(), C.data_ptr(), stream)
+                torch.cuda.synchronize()
+                assert np.array_equal(C.cpu().numpy(), oracle.classical(A.cpu().numpy(), B.cpu().numpy())), (n, call)
+        print("static-only-ok")
+    """)
+    r = subprocess.run([sys.executable, "-c", child], cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "static-only-ok" in r.stdout, r.stdout + r.stderr
