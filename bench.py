@@ -4,18 +4,20 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 A step is one whole product C = A.B (operand formation, the batched base products,
-recombination) on one batch of seeded synthetic input.  With N > 1 (torchrun, one rank per
-GPU) every rank runs an independent replica of the same product; there is no data-path
-collective.  Rank 0 prints ONE JSON line.  `--impl reference` times the CPU oracle on the
-host cores instead (a reported baseline, not a target).
+recombination) on one batch of seeded synthetic input.  With N > 1 every rank (one per GPU)
+runs an independent replica of the same product; there is no data-path collective.  Started
+without torchrun, `--gpus N` launches its own N ranks.  Rank 0 prints ONE JSON line; besides the
+headline workload it carries `per_config`, a short measurement of every configuration the
+metric is defined on.  `--impl reference` times the CPU oracle on the host cores instead (a
+reported baseline, not a target).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -38,15 +40,18 @@ WORKLOADS = {
     "gemm771x49": (771, 771, "", 49, "uniform", 6003, 0),
 }
 DEFAULT_WORKLOAD = "n4096"   # the configuration the headline metric is quoted on
+# the configurations of the metric, in the order they are reported in `per_config`, with their timed steps
+PER_CONFIG = (("n512", 200), ("n4096", 20), ("b32n2048", 10), ("n12345", 5), ("n16384", 5), ("n47040", 2))
 METRIC = "effective FP64 GFLOP/s (2n^3/t)"
 UNIT = "GFLOP/s"
 
-# DRAM bytes (read + write) of the dominant kernel's launch from one ncu capture, per workload
+# DRAM bytes (read + write) of the dominant kernel's launches per step, from one ncu capture of that workload
 # (profiles/gemm_f64_kernel_343x512.md); None where no capture of that exact launch exists.
 GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.125e9, "gemm512x343": 2.125e9}
 
 # FP64 arithmetic peak from unit counts and clocks: 148 SMs x 64 FP64 FMA lanes x 2 flop x 1.965 GHz
 FP64_PEAK_NOMINAL_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
+HBM_NOMINAL_GBS = 8000.0     # the figure the metric's definition names; the measured copy rate is the denominator used
 
 
 def describe(name):
@@ -63,13 +68,20 @@ def level_sizes(n, cutoff):
 
 
 def algorithmic_work(n, cutoff, batch):
-    """(base-product flops, sum/recombine bytes) one product must move: 7^L products of 2 m_L^3
-    flops; per node per level 16 h^2 words to form the sums + 11 h^2 to recombine."""
+    """(base-product flops, sum/recombine bytes) of one product with one streaming pass per level: 7^L
+    products of 2 m_L^3 flops; per node per level 16 h^2 words to form the sums + 11 h^2 to recombine."""
     m = level_sizes(n, cutoff)
     L = len(m) - 1
     f_base = batch * 7 ** L * 2.0 * m[-1] ** 3
     b_alg = batch * 8.0 * sum(7 ** i * 27 * m[i + 1] ** 2 for i in range(L))
     return f_base, b_alg
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
 
 
 class ClockSampler:
@@ -143,26 +155,216 @@ def whole_job_value(n, batch, ms_per_step, world):
     return world * 2.0 * n ** 3 * batch / (ms_per_step * 1e-3) / 1e9
 
 
+def free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def self_launch_command(gpus, argv):
+    """The command that runs this script as `gpus` ranks on this node (used when --gpus N > 1 is given
+    without a launcher): torch.distributed.run with a rendezvous on 127.0.0.1."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(gpus),
+            "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+
+
 def time_oracle_slab(n, A_host, B_host, target_seconds=12.0):
     """Time the classical oracle on a slab of rows of the same product; the slab is grown until it
-    costs about target_seconds.  Returns (GFLOP/s, rows, seconds)."""
+    costs about target_seconds.  Returns (GFLOP/s, rows, seconds, the slab of C)."""
     import oracle
     rows, t = min(n, 32), 0.0
     while True:
         t0 = time.perf_counter()
-        oracle.classical(A_host[:rows], B_host)
+        slab = oracle.classical(A_host[:rows], B_host)
         t = time.perf_counter() - t0
         if rows >= n or t >= target_seconds / 3:
             break
         rows = min(n, max(rows * 2, int(rows * 0.6 * target_seconds / max(t, 1e-3))))
-    return 2.0 * rows * n * n / t / 1e9, rows, t
+    return 2.0 * rows * n * n / t / 1e9, rows, t, slab
+
+
+def sample_indices(sizes, extra, seed):
+    """Row / column indices that touch every recursion boundary (first and last row of each quadrant at every
+    level, the peeled last row) plus seeded random ones."""
+    import numpy as np
+    n = sizes[0]
+    idx, starts = {0, n - 1}, [0]
+    for m, h in zip(sizes[:-1], sizes[1:]):
+        new = []
+        for s in starts[:32]:
+            for q in (0, 1):
+                o = s + q * h
+                new.append(o)
+                idx.update(i for i in (o, o + h - 1, o + h, s + m - 1) if 0 <= i < n)
+        starts = new
+    rng = np.random.default_rng(seed)
+    idx.update(int(i) for i in rng.integers(0, n, extra))
+    return np.array(sorted(idx), dtype=np.int64)
+
+
+def oracle_block_check(A, B, C, sizes, seed, exact):
+    """Part of the CPU-oracle leg: the block C[R, S] of the definition, computed by the classical oracle from
+    the sampled rows of A and columns of B, against the same block of the device result."""
+    import numpy as np
+    import torch
+    import oracle
+    R, S = sample_indices(sizes, 64, seed + 17), sample_indices(sizes, 64, seed + 29)
+    Rt, St = torch.from_numpy(R).to(A.device), torch.from_numpy(S).to(A.device)
+    rows = A.index_select(0, Rt).cpu().numpy()
+    cols = B.index_select(1, St).cpu().numpy()
+    got = C.index_select(0, Rt).index_select(1, St).cpu().numpy()
+    ref = oracle.classical(rows, cols)
+    if exact:
+        return bool(np.array_equal(got, ref))
+    return float(np.abs(got - ref).max())
+
+
+def absmax(X):
+    import torch
+    lo, hi = torch.aminmax(X)
+    return max(abs(float(lo)), abs(float(hi)))
+
+
+def timed_steps(fn, steps, stream, barrier=None):
+    """K steps in one timed region with a CUDA event between consecutive steps (no host synchronisation inside):
+    returns the per-step intervals in ms and the wall-clock bracket of the region."""
+    import torch
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    w0 = time.time()
+    events[0].record(stream)
+    for i in range(steps):
+        fn()
+        events[i + 1].record(stream)
+    if barrier:
+        barrier()
+    else:
+        torch.cuda.synchronize()
+    w1 = time.time()
+    return [events[i].elapsed_time(events[i + 1]) for i in range(steps)], events[0].elapsed_time(events[steps]) / steps, w0, w1
+
+
+def measure(name, steps, warmup, rank, world, dev, sampler_factory=None, want_cublas=True, want_oracle=True):
+    """One configuration on this rank's GPU: the timed region (K steps, one CUDA event between steps, barrier and
+    synchronize on both sides), a second pass with per-kernel-family events, cuBLAS DGEMM on the same buffers,
+    and -- in the CPU-oracle leg -- a sampled block of the definition on the float and the integer variant."""
+    import torch
+    import torch.distributed as dist
+    from paper_1202_3173_b200 import Plan, inputs
+
+    n, cutoff, sched, batch, dist_name, seed, budget = WORKLOADS[name]
+    if budget < 0:
+        budget = int(min(180e9, torch.cuda.mem_get_info()[0] - 4e9) - 3 * n * n * 8)
+    A, B = inputs.pair(n, dist_name, seed + 1000 * rank, device=dev, batch=None if batch == 1 else batch)
+    C = torch.empty_like(A)
+    plan = Plan(n, cutoff, sched, batch=batch, workspace_budget_bytes=budget)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        plan(A, B, out=C)
+    barrier()
+    sampler = sampler_factory() if sampler_factory else None
+    per_step, ms_mean_local, w0, w1 = timed_steps(lambda: plan(A, B, out=C), steps, stream, barrier)
+    clocks = sampler.stop(w0, w1) if sampler else None
+    ms_median_local = statistics.median(per_step)
+    ms = reduce_max(ms_median_local, dev)
+    ms_mean = reduce_max(ms_mean_local, dev)
+
+    # per-kernel-family split: a separate, shorter pass with two events around every launch
+    split_steps = max(1, min(steps, 5))
+    plan.set_timing(True)
+    for _ in range(split_steps):
+        plan(A, B, out=C)
+    kinds = {k: v / split_steps for k, v in plan.timings_ms().items()}
+    plan.set_timing(False)
+
+    sizes = plan.level_sizes
+    f_base, b_27 = algorithmic_work(n, sizes[-1], batch)
+    pass_bytes = plan.pass_bytes
+    hbm_gbs, hbm_src = hbm_peak()
+    product_kind = "fused_step" if kinds.get("fused_step", 0.0) > 0 else "gemm"
+    product_ms = kinds[product_kind]
+    add_ms = sum(v for k, v in kinds.items() if k not in ("gemm", "fused_step", "scale"))
+    out = {
+        "workload": name, "n": n, "batch": batch, "schedule": plan.schedule, "levels": sizes,
+        "workspace_bytes": plan.workspace_bytes, "steps": steps, "launches_per_step": plan.launch_count,
+        "launches_by_kind": {k: v for k, v in plan.launches_by_kind().items() if v},
+        "ms_per_step": ms, "ms_per_step_mean": ms_mean, "ms_per_step_min": min(per_step), "ms_per_step_max": max(per_step),
+        "effective_gflops": whole_job_value(n, batch, ms, 1),
+        "actual_gflops": (f_base + 15 * b_27 / (27 * 8)) / (ms * 1e-3) / 1e9,
+        "kernel_ms_per_step": {k: round(v, 6) for k, v in kinds.items() if v},
+        "product_kernel": product_kind,
+        "product_tflops": f_base / (product_ms * 1e-3) / 1e12 if product_ms > 0 else None,
+        "product_frac_of_fp64_peak": f_base / (product_ms * 1e-3) / 1e12 / FP64_PEAK_NOMINAL_TFLOPS if product_ms > 0 else None,
+        "add_bytes_scheduled": pass_bytes, "add_bytes_27h2": b_27,
+        "add_gbs": pass_bytes / (add_ms * 1e-3) / 1e9 if add_ms > 0 else None,
+        "add_frac_of_measured_hbm": pass_bytes / (add_ms * 1e-3) / 1e9 / hbm_gbs if add_ms > 0 else None,
+        "add_frac_of_nominal_8000": pass_bytes / (add_ms * 1e-3) / 1e9 / HBM_NOMINAL_GBS if add_ms > 0 else None,
+        "l2": "inputs larger than L2 (A+B+C %.0f MB + workspace): no flush" % (3 * batch * n * n * 8 / 1e6)
+              if 3 * batch * n * n * 8 > 126e6 else
+              "L2-resident by nature (A+B+C %.1f MB): launch-bound, no flush between steps" % (3 * batch * n * n * 8 / 1e6),
+    }
+    # roofline of the whole product: base products at the FP64 peak + the scheduled passes at the HBM rate; and the
+    # floor no fusion can beat (products at peak + A and B read, C written once)
+    t_roof = (f_base / (FP64_PEAK_NOMINAL_TFLOPS * 1e12) + pass_bytes / (hbm_gbs * 1e9)) * 1e3
+    t_floor = (f_base / (FP64_PEAK_NOMINAL_TFLOPS * 1e12) + 3.0 * batch * n * n * 8 / (hbm_gbs * 1e9)) * 1e3
+    t_27 = (f_base / (FP64_PEAK_NOMINAL_TFLOPS * 1e12) + b_27 / (hbm_gbs * 1e9)) * 1e3
+    out["path_roofline"] = {"t_roof_ms": t_roof, "frac": t_roof / ms_median_local,
+                            "bytes": "the passes as scheduled (strassen_plan_pass_bytes): multi-level passes, DFS surcharge and peeling included",
+                            "floor_ms": t_floor, "frac_of_floor": t_floor / ms_median_local,
+                            "floor": "base products at the FP64 peak + 3 n^2 words over HBM: what no fusion of the passes can beat",
+                            "t_one_pass_per_level_ms": t_27, "ratio_to_one_pass_per_level": t_27 / ms_median_local,
+                            "one_pass_per_level": "27 h^2 words per node per level; NOT a lower bound: multi-level passes move less, "
+                                                  "so this ratio may exceed 1",
+                            "base_flops": f_base, "hbm_gbs": hbm_gbs, "hbm_source": hbm_src}
+
+    if want_cublas:
+        Cc = C if 3 * batch * n * n * 8 > 40e9 else torch.empty_like(A)      # no room for a fourth matrix at the largest size
+        reps = max(2, min(steps, 20 if n <= 4096 else 5))
+        try:
+            for _ in range(3 if n <= 16384 else 1):
+                torch.matmul(A, B, out=Cc)
+            torch.cuda.synchronize()
+            c_steps, c_mean, _, _ = timed_steps(lambda: torch.matmul(A, B, out=Cc), reps, stream)     # same protocol as ours
+            cms = statistics.median(c_steps)
+            out["cublas_dgemm"] = {"ms": cms, "ms_mean": c_mean, "steps": reps, "gflops": 2.0 * n ** 3 * batch / (cms * 1e-3) / 1e9}
+            out["vs_cublas"] = cms / ms_median_local
+        except Exception as exc:
+            out["cublas_dgemm"] = {"error": str(exc)[:200]}
+        if Cc is C:
+            plan(A, B, out=C)               # C holds our product again
+            torch.cuda.synchronize()
+        del Cc
+
+    if want_oracle and rank == 0:
+        # CPU-oracle leg, parity part: a block of the definition that contains every recursion boundary
+        try:
+            a0, b0, c0 = (A, B, C) if batch == 1 else (A[0], B[0], C[0])
+            lim = 1e-11 * n * absmax(A) * absmax(B)
+            err = oracle_block_check(a0, b0, c0, sizes, seed, exact=False)
+            out["max_err"], out["bound"], out["err_over_bound"] = err, lim, err / lim
+            del A, B, a0, b0, c0
+            A, B = inputs.pair(n, "int8", seed + 500, device=dev, batch=None if batch == 1 else batch)
+            plan(A, B, out=C)
+            torch.cuda.synchronize()
+            a0, b0, c0 = (A, B, C) if batch == 1 else (A[0], B[0], C[0])
+            out["int_equal"] = oracle_block_check(a0, b0, c0, sizes, seed + 500, exact=True)
+            del a0, b0, c0
+        except Exception as exc:
+            out["oracle_check_error"] = str(exc)[:200]
+    return out, clocks, plan, (A, B, C)
 
 
 def run_reference(args, rank, world):
     """The reference arm: the CPU oracle as it stands, on the host cores, rank 0 only."""
     if rank != 0:
         return
-    import numpy as np
     import oracle
     from paper_1202_3173_b200 import inputs
     n, cutoff, sched, batch, dist_name, seed, _ = WORKLOADS[args.workload]
@@ -194,14 +396,26 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
-    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg (and its parity samples)")
     ap.add_argument("--no-cublas", action="store_true", help="skip the cuBLAS DGEMM comparator")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-probes", action="store_true", help="skip the FP64 rate probes")
     ap.add_argument("--no-autotune", action="store_true", help="skip the measured choice of steps and interleaving")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short measurement of the other configurations")
     ap.add_argument("--graph", action="store_true", help="also time the plan replayed as one CUDA graph")
+    ap.add_argument("--check-launch", action="store_true",
+                    help="no GPU work: every rank joins a gloo group and exchanges a stand-in time through the same reduction "
+                         "(checks the launcher plumbing of --gpus N on a machine without GPUs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher around us: build first (no rank may find a half-linked library), then become N ranks
+        if args.impl == "ours" and not args.check_launch:
+            from paper_1202_3173_b200 import build as _build
+            _build.ensure_built()
+        cmd = self_launch_command(args.gpus, sys.argv[1:])
+        os.execvp(cmd[0], cmd)
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -210,59 +424,59 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank, world)
         return
+    if args.check_launch:
+        import torch
+        import torch.distributed as dist
+        if world > 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            dist.init_process_group("gloo")
+        ms = reduce_max(3.0 + rank, torch.device("cpu"))       # stand-in per-rank times 3, 4, ... ms
+        if rank == 0:
+            print(json.dumps({"check_launch": True, "n_gpus": world, "ms_per_step": ms, "scaling": "weak",
+                              "value": whole_job_value(*WORKLOADS[args.workload][:1], WORKLOADS[args.workload][3], ms, world)}),
+                  flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     import torch
     import torch.distributed as dist
-    from paper_1202_3173_b200 import build as _build
-    if local_rank == 0:
-        _build.ensure_built()
-    from paper_1202_3173_b200 import Plan, binding, inputs
-
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("NCCL_DEBUG", "INFO")          # the communicator log shows every rank that joined
         dist.init_process_group("nccl", device_id=dev)
+    from paper_1202_3173_b200 import build as _build
+    if local_rank == 0:
+        _build.ensure_built()                                 # one rank (re)builds; the others wait, then load
+    if world > 1:
+        dist.barrier()
+    from paper_1202_3173_b200 import Plan, binding
 
-    n, cutoff, sched, batch, dist_name, seed, budget = WORKLOADS[args.workload]
-    if budget < 0:
-        budget = int(min(180e9, torch.cuda.mem_get_info()[0] - 4e9) - 3 * n * n * 8)
-    A, B = inputs.pair(n, dist_name, seed + 1000 * rank, device=dev, batch=None if batch == 1 else batch)
-    C = torch.empty_like(A)
-    plan = Plan(n, cutoff, sched, batch=batch, workspace_budget_bytes=budget)
+    n, cutoff, sched, batch, dist_name, seed, _ = WORKLOADS[args.workload]
+    head, clocks, plan, (A, B, C) = measure(args.workload, args.steps, args.warmup, rank, world, dev,
+                                            sampler_factory=(lambda: ClockSampler(local_rank)) if rank == 0 else None,
+                                            want_cublas=rank == 0 and not args.no_cublas,
+                                            want_oracle=rank == 0 and not args.no_cpu_baseline)
     stream = torch.cuda.current_stream()
+    ms = head["ms_per_step"]
+    sched_resolved = plan.schedule
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing -----------------------------------------------------------
-    for _ in range(args.warmup):
-        plan(A, B, out=C)
-    barrier()
-    plan.set_timing(True)
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    w0 = time.time()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        plan(A, B, out=C)
-    ev1.record(stream)
-    barrier()
-    w1 = time.time()
-    clocks = sampler.stop(w0, w1) if sampler else None
-    ms_local = ev0.elapsed_time(ev1) / args.steps
-    kinds = plan.timings_ms()
-    plan.set_timing(False)
-    ms = reduce_max(ms_local, dev)
-
-    sched_resolved = plan.schedule
+    del A, B
+    from paper_1202_3173_b200 import inputs
+    A, B = inputs.pair(n, dist_name, seed + 1000 * rank, device=dev, batch=None if batch == 1 else batch)
     hA = hB = None
     if not args.no_e2e or (rank == 0 and not args.no_cpu_baseline):
         hA, hB = A.cpu().pin_memory(), B.cpu().pin_memory()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def run_e2e():
         """Host buffers, copies inside the timed region.  Runs last: the device copies of A, B, C are freed
@@ -303,45 +517,20 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- rank 0: comparator, probes, CPU oracle, report ----------------------------------------
-    f_base, b_alg = algorithmic_work(n, cutoff, batch)
-    gemm_launches = plan.launches_by_kind()["gemm"]
-    gemm_ms = kinds["gemm"] / (args.steps * gemm_launches)
-    achieved_tflops = f_base / gemm_launches / (gemm_ms * 1e-3) / 1e12
-
+    # ---- rank 0: probes, tuner, CPU oracle, the other configurations, report --------------------
+    f_base, _ = algorithmic_work(n, head["levels"][-1], batch)
     probes = {}
-    for kind, name in enumerate(("dfma", "dmma_m8n8k4", "dmma_m16n8k4", "dmma_m16n8k8", "dmma_m16n8k16")):
+    for kind, pname in enumerate(("dfma", "dmma_m8n8k4", "dmma_m16n8k4", "dmma_m16n8k8", "dmma_m16n8k16")):
         if args.no_probes:
             break
         try:
-            probes[name] = round(binding.strassen_probe_fp64(kind, 20000, stream.cuda_stream), 2)
+            probes[pname] = round(binding.strassen_probe_fp64(kind, 20000, stream.cuda_stream), 2)
         except Exception as exc:   # a probe is context, never fatal
-            probes[name] = str(exc)
-    fp64_measured = max([v for v in probes.values() if isinstance(v, float)] or [FP64_PEAK_NOMINAL_TFLOPS])
-
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        hbm_gbs, hbm_src = json.load(open(peaks_path))["hbm_gbs"], "measured"
-    else:
-        hbm_gbs, hbm_src = 6650.0, "fallback"
-    t_roof_ms = (f_base / (FP64_PEAK_NOMINAL_TFLOPS * 1e12) + b_alg / (hbm_gbs * 1e9)) * 1e3
-
-    cublas = None
-    if not args.no_cublas:
-        Cc = torch.empty_like(A)
-        for _ in range(3):
-            torch.matmul(A, B, out=Cc)
-        torch.cuda.synchronize()
-        reps = max(3, min(args.steps, 10))
-        ev0.record(stream)
-        for _ in range(reps):
-            torch.matmul(A, B, out=Cc)
-        ev1.record(stream)
-        torch.cuda.synchronize()
-        cms = ev0.elapsed_time(ev1) / reps
-        cublas = {"ms": cms, "gflops": 2.0 * n ** 3 * batch / (cms * 1e-3) / 1e9,
-                  "max_abs_diff_vs_ours": float((Cc - C).abs().max()) if n <= 16384 else None}
-        del Cc
+            probes[pname] = str(exc)
+    measured = [v for v in probes.values() if isinstance(v, float)]
+    fp64_peak, peak_source = ((max(measured), "strassen_probe_fp64 in this run: register-resident mma.sync f64 loop on every SM")
+                              if measured else
+                              (FP64_PEAK_NOMINAL_TFLOPS, "148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz (unit counts and max clock)"))
 
     tuned = None
     if not args.no_autotune:
@@ -381,27 +570,74 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
+        import numpy as np
         import oracle
         a_h = (hA if batch == 1 else hA[0]).numpy()
         b_h = (hB if batch == 1 else hB[0]).numpy()
-        g, rows, secs = time_oracle_slab(n, a_h, b_h)
+        g, rows, secs, slab = time_oracle_slab(n, a_h, b_h)
+        plan(A, B, out=C)
+        torch.cuda.synchronize()
+        ours = (C if batch == 1 else C[0])[:rows].cpu().numpy()
+        slab_err = float(np.abs(ours - slab).max())
         cpu = {"value": g, "unit": UNIT, "cores": oracle.cores(), "kind": "oracle",
-               "sample": "classical oracle on the first %d of %d rows of one product (%.1f s); classical flops "
-                         "equal effective flops, so the rate stands for the whole product" % (rows, n, secs)}
+               "sample": "classical oracle (the definition, Oracle A) on the first %d of %d rows of one product (%.1f s); "
+                         "classical flops equal effective flops, so the rate stands for the whole product" % (rows, n, secs),
+               "max_err_on_sample": slab_err, "bound": head.get("bound")}
+        # Oracle B, the CPU Strassen-Winograd with the same cutoff, timed once on a leading block it finishes in seconds
+        try:
+            nb = n if n <= 4096 else 4096
+            t0 = time.perf_counter()
+            cb, counters = oracle.strassen_winograd(np.ascontiguousarray(a_h[:nb, :nb]), np.ascontiguousarray(b_h[:nb, :nb]),
+                                                    head["levels"][-1])
+            tb = time.perf_counter() - t0
+            cpu["strassen_winograd_oracle"] = {
+                "value": 2.0 * nb ** 3 / tb / 1e9, "unit": "effective " + UNIT, "seconds": tb, "n": nb,
+                "cutoff": head["levels"][-1], "base_products": int(counters["base_calls"]),
+                "sample": "Oracle B on the leading %d x %d blocks of A and B, once" % (nb, nb)}
+        except Exception as exc:
+            cpu["strassen_winograd_oracle"] = {"error": str(exc)[:200]}
 
-    launches_by_kind, launch_count, level_list, ws_bytes = (plan.launches_by_kind(), plan.launch_count, plan.level_sizes,
-                                                        plan.workspace_bytes)
+    launch_count = plan.launch_count
     (e2e_ms, e2e_pipe_ms), e2e_error = run_e2e()
+    plan.close()
+    del plan
+    torch.cuda.empty_cache()
+
+    per_config = []
+    if not args.no_per_config and args.workload == DEFAULT_WORKLOAD and world == 1:
+        for cname, csteps in PER_CONFIG:
+            if cname == args.workload:
+                per_config.append(dict(head, note="the headline run above"))
+                continue
+            cn, _, _, cb, _, _, cbudget = WORKLOADS[cname]
+            need = 3 * cb * cn * cn * 8 + (110e9 if cbudget < 0 else 45e9 if cbudget else 16e9)
+            torch.cuda.empty_cache()
+            if torch.cuda.mem_get_info()[0] < need:
+                per_config.append({"workload": cname, "skipped": "needs about %.0f GB of free device memory" % (need / 1e9)})
+                continue
+            try:
+                res, _, cplan, bufs = measure(cname, csteps, 3, 0, 1, dev, want_cublas=not args.no_cublas,
+                                              want_oracle=not args.no_cpu_baseline)
+                cplan.close()
+                del cplan, bufs
+                per_config.append(res)
+            except Exception as exc:
+                per_config.append({"workload": cname, "error": str(exc)[:300]})
+            torch.cuda.empty_cache()
+
+    product_kind = head["product_kernel"]
+    product_ms = head["kernel_ms_per_step"].get(product_kind)
+    achieved = head["product_tflops"]
     ours_gflops = whole_job_value(n, batch, ms, world)
     line = {
         "metric": METRIC, "value": ours_gflops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "ms_per_step": ms, "ms_per_step_mean": head["ms_per_step_mean"],
+        "timing": "median of the %d per-step CUDA-event intervals of one timed region (barrier + synchronize on both sides, "
+                  "no per-launch events inside); max over ranks" % args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": describe(args.workload), "schedule": sched_resolved, "levels": level_list,
-                   "workspace_bytes": ws_bytes,
-                   "l2": "inputs larger than L2 (A+B+C %.0f MB + workspace)" % (3 * batch * n * n * 8 / 1e6)
-                         if 3 * batch * n * n * 8 > 126e6 else "L2-resident problem (A+B+C %.1f MB): launch-bound"
-                         % (3 * batch * n * n * 8 / 1e6),
+        "config": {"workload": describe(args.workload), "schedule": sched_resolved, "levels": head["levels"],
+                   "workspace_bytes": head["workspace_bytes"], "l2": head["l2"],
                    "parallelism": "replicas only (no collective)" if world > 1 else "single GPU"},
         "clocks": clocks,
         "e2e_error": e2e_error,
@@ -413,24 +649,34 @@ def main():
                 "h2d_bytes_per_step": 2 * batch * n * n * 8, "d2h_bytes_per_step": batch * n * n * 8,
                 "in_order_ms_per_step": e2e_ms, "pipelined_ms_per_step": e2e_pipe_ms},
         "gpu_launches": args.steps * launch_count,
-        "roofline": {"bound": "alu", "kernel": "gemm_f64_kernel (batched base products)", "achieved": achieved_tflops,
-                     "peak": FP64_PEAK_NOMINAL_TFLOPS, "unit": "TFLOP/s", "frac": achieved_tflops / FP64_PEAK_NOMINAL_TFLOPS,
-                     "peak_source": "148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz (unit counts and max clock)",
-                     "fp64_probe_tflops": probes, "frac_of_probe": achieved_tflops / fp64_measured,
-                     "ms_per_launch": gemm_ms, "flops_per_launch": f_base / gemm_launches,
-                     "traffic": GEMM_DRAM_TRAFFIC_BYTES.get(args.workload)},
-        "path_roofline": {"t_roof_ms": t_roof_ms, "frac": t_roof_ms / ms_local, "base_flops": f_base, "add_bytes": b_alg,
-                          "hbm_gbs": hbm_gbs, "hbm_source": hbm_src,
-                          "kernel_ms_per_step": {k: v / args.steps for k, v in kinds.items()}},
-        "actual_gflops": (f_base + 15 * b_alg / (27 * 8)) / (ms * 1e-3) / 1e9 * world,
+        "roofline": {"bound": "alu",
+                     "kernel": "gemm_f64_kernel (batched base products)" if product_kind == "gemm"
+                               else "fused_step_kernel (sums, seven products and U-chain of the deepest step)",
+                     "achieved": achieved, "peak": fp64_peak, "unit": "TFLOP/s", "frac": achieved / fp64_peak if achieved else None,
+                     "peak_source": peak_source,
+                     "peak_nominal": FP64_PEAK_NOMINAL_TFLOPS, "frac_of_nominal": achieved / FP64_PEAK_NOMINAL_TFLOPS if achieved else None,
+                     "fp64_probe_tflops": probes,
+                     "flops_per_step": f_base, "kernel_ms_per_step": product_ms,
+                     "launches_per_step": head["launches_by_kind"].get(product_kind),
+                     "launches": "the family's launches of one step are timed together (two CUDA events around each, a separate "
+                                 "pass from the timed region); at n=4096 they are 342 leaves on 128 x 128 tiles and 1 leaf on "
+                                 "64 x 64 tiles",
+                     "traffic": GEMM_DRAM_TRAFFIC_BYTES.get(args.workload),
+                     "traffic_source": "one ncu capture of this launch (profiles/), per step; not measured in this run"
+                                       if GEMM_DRAM_TRAFFIC_BYTES.get(args.workload) else None},
+        "path_roofline": dict(head["path_roofline"], kernel_ms_per_step=head["kernel_ms_per_step"]),
+        "add_kernels": {k: head[k] for k in ("add_bytes_scheduled", "add_bytes_27h2", "add_gbs", "add_frac_of_measured_hbm",
+                                             "add_frac_of_nominal_8000")},
+        "actual_gflops": head["actual_gflops"] * world,
+        "parity": {k: head.get(k) for k in ("max_err", "bound", "err_over_bound", "int_equal")},
         "autotuned": tuned,
         "cuda_graph_ms_per_step": graph_ms,
-        "cublas_dgemm": cublas,
-        "vs_cublas": (cublas["ms"] / ms_local) if cublas else None,
+        "cublas_dgemm": head.get("cublas_dgemm"),
+        "vs_cublas": head.get("vs_cublas"),
         "cpu_baseline": cpu,
+        "per_config": per_config,
     }
     print(json.dumps(line), flush=True)
-    plan.close()
     if world > 1:
         dist.destroy_process_group()
 

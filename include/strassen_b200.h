@@ -63,7 +63,8 @@ typedef enum strassen_kernel_kind {
     STRASSEN_K_ACCUMULATE = 4, /* DFS fold of one Q_j into the quadrants of C                       */
     STRASSEN_K_PEEL = 5,       /* peeling fix-ups: rank-one update, last column, last row           */
     STRASSEN_K_SCALE = 6,      /* diagonal scaling passes (STRASSEN_FLAG_SCALE_*)                   */
-    STRASSEN_K_COUNT = 7
+    STRASSEN_K_FUSED_STEP = 7, /* a whole BFS step of the deepest level (sums, products, U-chain) in one kernel */
+    STRASSEN_K_COUNT = 8
 } strassen_kernel_kind;
 
 /* Extended plan description.  Zero-initialise, then set what differs from the default. */
@@ -85,6 +86,16 @@ typedef struct strassen_options {
  * pass per level, TWO_LEVEL_PASSES at most two levels per pass. */
 #define STRASSEN_FLAG_SINGLE_LEVEL_PASSES 1
 #define STRASSEN_FLAG_TWO_LEVEL_PASSES 32
+
+/* The deepest recursion level, when it is a BFS step, can run as ONE kernel that forms the operand
+ * sums in registers while it loads the quadrants of A and B, accumulates the seven products side by
+ * side on the FP64 tensor cores and applies the U-chain before it stores C [Section 6.3 "Optimizing
+ * on-node performance" asks for such a shared-memory Strassen; Appendix A for the step]: same
+ * operations in the same order as the three-launch path, bit-identical results, no workspace traffic
+ * for that level.  By default the library uses it where the base products are too few to fill the
+ * GPU (small n); FUSED_STEP uses it whenever the deepest level is a BFS step, NO_FUSED_STEP never. */
+#define STRASSEN_FLAG_FUSED_STEP 64
+#define STRASSEN_FLAG_NO_FUSED_STEP 128
 
 /* Replay the plan's launch list as one CUDA graph: the first strassen_dgemm call with a given
  * (A, B, C, workspace) captures the launches on an internal stream and instantiates the graph; that
@@ -196,6 +207,17 @@ int64_t strassen_plan_base_products(const strassen_plan *plan);         /* batch
 int64_t strassen_plan_launch_count(const strassen_plan *plan);          /* kernels per strassen_dgemm (counted
                                                                            for a 148-SM device)       */
 int64_t strassen_plan_launches_of(const strassen_plan *plan, int kind); /* ... of one family          */
+
+/* Bytes the plan's streaming passes move per product as scheduled: operand formation and recombination
+ * of every BFS step (a pass over two or three levels counted with what it really reads and writes, less
+ * than one pass per level), formation and fold of every DFS step, the peeled last column and row of
+ * odd sizes.  The base products' own operand traffic is not included.  This is the HBM term of the
+ * path's roofline [Section 3.3.1 counts the additions of a step; on a GPU they are bound by the bytes]. */
+double strassen_plan_pass_bytes(const strassen_plan *plan);
+
+/* The cost model's estimate of one product in milliseconds on a B200 (the estimate that orders
+ * strassen_autotune's search and picks plans created with cutoff 0).  Measurement aid. */
+double strassen_plan_model_ms(const strassen_plan *plan);
 
 /* Workspace (bytes, unpadded) a schedule string needs under the paper's accounting of 21
  * quarter-size matrices per BFS parent and 3 per DFS parent [Sections 3.3.1, 3.4.1], or,

@@ -65,6 +65,15 @@ class Plan:
         return self._ws
 
     @property
+    def pass_bytes(self):
+        """HBM bytes the streaming passes (sums, recombination, DFS folds, peeling) move per product as scheduled."""
+        return binding.strassen_plan_pass_bytes(self._h)
+
+    @property
+    def model_ms(self):
+        return binding.strassen_plan_model_ms(self._h)
+
+    @property
     def launch_count(self):
         return binding.strassen_plan_launch_count(self._h)
 

@@ -19,10 +19,12 @@ STRASSEN_FLAG_HOST_PIPELINE = 4
 STRASSEN_FLAG_SCALE_OUTSIDE = 8
 STRASSEN_FLAG_SCALE_INSIDE = 16
 STRASSEN_FLAG_TWO_LEVEL_PASSES = 32
+STRASSEN_FLAG_FUSED_STEP = 64
+STRASSEN_FLAG_NO_FUSED_STEP = 128
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SCHEDULE", -3: "WORKSPACE_TOO_SMALL", -4: "ALIAS",
                 -5: "MISALIGNED", -6: "CUDA_ERROR", -7: "OUT_OF_MEMORY"}
-K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_SCALE, K_COUNT = range(8)
-KERNEL_KINDS = ("form", "gemm", "recombine", "form_one", "accumulate", "peel", "scale")
+K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_SCALE, K_FUSED_STEP, K_COUNT = range(9)
+KERNEL_KINDS = ("form", "gemm", "recombine", "form_one", "accumulate", "peel", "scale", "fused_step")
 
 # every symbol the header declares: (name, restype, argtypes)
 _vp, _i64, _sz, _cp, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_char_p, ctypes.c_int
@@ -65,6 +67,8 @@ SYMBOLS = [
     ("strassen_plan_base_products", _i64, [_vp]),
     ("strassen_plan_launch_count", _i64, [_vp]),
     ("strassen_plan_launches_of", _i64, [_vp, _int]),
+    ("strassen_plan_pass_bytes", ctypes.c_double, [_vp]),
+    ("strassen_plan_model_ms", ctypes.c_double, [_vp]),
     ("strassen_schedule_model_bytes", _sz, [_i64, _i64, _i64, _cp, _int]),
     ("strassen_plan_set_timing", _int, [_vp, _int]),
     ("strassen_plan_get_timings", _int, [_vp, _dp]),
@@ -178,6 +182,14 @@ def strassen_plan_launch_count(plan: int) -> int:
 
 def strassen_plan_launches_of(plan: int, kind: int) -> int:
     return lib().strassen_plan_launches_of(plan, kind)
+
+
+def strassen_plan_pass_bytes(plan: int) -> float:
+    return lib().strassen_plan_pass_bytes(plan)
+
+
+def strassen_plan_model_ms(plan: int) -> float:
+    return lib().strassen_plan_model_ms(plan)
 
 
 def strassen_schedule_model_bytes(n, cutoff, batch, schedule, accounting=21) -> int:

@@ -56,8 +56,8 @@ struct strassen_plan {
     cudaStream_t capture_stream = nullptr;
     cudaGraphExec_t graph_exec = nullptr;
     const void *graph_ptrs[4] = {nullptr, nullptr, nullptr, nullptr};   // A, B, C, workspace the graph was captured for
-    double acc_ms[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0, 0};
-    int64_t launches[STRASSEN_K_COUNT] = {0, 0, 0, 0, 0, 0, 0};
+    double acc_ms[STRASSEN_K_COUNT] = {};
+    int64_t launches[STRASSEN_K_COUNT] = {};
     int64_t launch_total = 0;
 };
 
@@ -69,6 +69,7 @@ int family(int op_kind)
     if (op_kind == OP_FORM2 || op_kind == OP_FORM3) return STRASSEN_K_FORM;
     if (op_kind == OP_RECOMBINE2 || op_kind == OP_RECOMBINE3) return STRASSEN_K_RECOMBINE;
     if (op_kind == OP_SCALE_IN || op_kind == OP_SCALE_OUT) return STRASSEN_K_SCALE;
+    if (op_kind == OP_FUSED_STEP) return STRASSEN_K_FUSED_STEP;
     return op_kind;
 }
 
@@ -130,6 +131,7 @@ int ensure_device_state(strassen_plan *p, cudaStream_t stream)
         e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
         e = configure_gemm_kernels();       // opt-in to large dynamic shared memory, outside any capture
+        if (e == cudaSuccess) e = configure_fused_step_kernels();
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute");
         p->device = dev;
     } else {
@@ -201,6 +203,7 @@ int enqueue_launches(strassen_plan *p, const Bases &bases, bool bases16, cudaStr
         case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
         case OP_FORM3: e = launch_form3(p->d_tab, op, bases, stream, &launched); break;
         case OP_RECOMBINE3: e = launch_recombine3(p->d_tab, op, bases, stream, &launched); break;
+        case OP_FUSED_STEP: e = launch_fused_step(p->d_tab, op, bases, p->sm_count, stream, &launched); break;
         case OP_SCALE_IN: e = launch_scale_in(p->d, bases, stream, &launched); break;
         case OP_SCALE_OUT: e = launch_scale_out(p->d, bases, stream, &launched); break;
         }
@@ -286,6 +289,7 @@ strassen_plan *create(const strassen_options &o)
         delete p;
         return nullptr;
     }
+    d.fused_step = (o.flags & STRASSEN_FLAG_NO_FUSED_STEP) ? 2 : (o.flags & STRASSEN_FLAG_FUSED_STEP) ? 1 : 0;
     d.max_fused_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) ? 1 : (o.flags & STRASSEN_FLAG_TWO_LEVEL_PASSES) ? 2 : 3;
     p->use_graph = (o.flags & STRASSEN_FLAG_CUDA_GRAPH) != 0;
     p->host_pipeline = (o.flags & STRASSEN_FLAG_HOST_PIPELINE) != 0;
@@ -309,7 +313,7 @@ strassen_plan *create(const strassen_options &o)
     if (cutoff == 0 && want_auto) {
         // number of steps and interleaving by the cost model, among everything that fits the budget; bases
         // below 256 are left out: there the passes are latency-bound and the model, built on rates, is too kind
-        if (!model_choice(n, batch, int64_t(budget / 8), 256, &d.sizes, &d.schedule)) {
+        if (!model_choice(n, batch, int64_t(budget / 8), 256, d.fused_step, &d.sizes, &d.schedule)) {
             fail(STRASSEN_WORKSPACE_TOO_SMALL, "no plan fits the workspace budget");
             delete p;
             return nullptr;
@@ -577,6 +581,7 @@ int64_t strassen_plan_base_products(const strassen_plan *p)
     int64_t c = 0;
     for (const Launch &op : p->d.launches)
         if (op.kind == OP_GEMM) c += op.count;
+        else if (op.kind == OP_FUSED_STEP) c += 7 * op.count;     // the seven products of each parent, inside the kernel
     return c;
 }
 int64_t strassen_plan_launch_count(const strassen_plan *p) { return p ? p->launch_total : -1; }
@@ -584,6 +589,18 @@ int64_t strassen_plan_launches_of(const strassen_plan *p, int kind)
 {
     if (!p || kind < 0 || kind >= STRASSEN_K_COUNT) return -1;
     return p->launches[kind];
+}
+
+double strassen_plan_pass_bytes(const strassen_plan *p)
+{
+    if (!p) return -1.0;
+    return plan_model_parts(p->d.sizes, p->d.schedule, p->d.batch, p->d.fused_step).pass_bytes;
+}
+
+double strassen_plan_model_ms(const strassen_plan *p)
+{
+    if (!p) return -1.0;
+    return plan_model_ms(p->d.sizes, p->d.schedule, p->d.batch, p->d.fused_step);
 }
 
 size_t strassen_schedule_model_bytes(int64_t n, int64_t cutoff, int64_t batch, const char *schedule, int accounting)

@@ -1,0 +1,358 @@
+// One whole Strassen-Winograd step in a single kernel (Appendix A; Algorithm 1 with its three
+// "locally compute" lines collapsed): C = A.B for parents of size 2h (+1 when peeled) straight from
+// the quadrants of A and B, with no operand sums, no products and no node table for the children
+// ever reaching memory.
+//
+// A CTA owns a tile of positions (r, c) of the h x h quadrant grid and computes all seven
+// products Q_0..Q_6 at those positions at once:
+//   * the loader stages, per 16-deep slab, the tile's rows of the four quadrants of A and the
+//     tile's columns of the four quadrants of B (cp.async ring, as in the base-product kernel);
+//   * a warp reads the four quadrant fragments of each side from shared memory and forms the seven
+//     operand fragments in registers (T2 = A21 + A22, T3 = T2 - A11, T4 = A11 - A21, T5 = A12 - T3;
+//     S2 = B12 - B11, S3 = B22 - S2, S4 = B22 - B12, S6 = S3 - B21): four adds instead of three more
+//     loads per side;
+//   * seven FP64 tensor-core accumulator sets (mma.sync m8n8k4), one per product, k ascending;
+//   * the epilogue runs the U-chain (U1 = Q0 + Q3, U2 = U1 + Q4, U3 = U1 + Q2; C11 = Q0 + Q1,
+//     C12 = U3 + Q5, C21 = U2 - Q6, C22 = U2 + Q2) in registers and stores the four quadrants of C,
+//     with the rank-one term of a peeled (odd-size) parent added on the way out.
+// The operations on every element are those of the three-launch path (formation, base products,
+// recombination) in the same order, so the results have the same bits.
+//
+// What it costs: every CTA re-reads its row panel of A and column panel of B, so the operands cross
+// L2 -> SM about (h / tile) times instead of once, and the seven accumulator sets cap the warp tile
+// at 16 x 16 positions.  It pays where the three-launch path is bound by launches and by tiles too
+// few to fill the SMs (small n), not where the base products already run near the FP64 peak.
+#include "kernels.h"
+
+namespace strassen {
+
+namespace {
+
+template <int WARPS_M_, int WARPS_N_, int MT_, int NT_, int BK_, int STAGES_, int CTAS_, bool DOUBLE_BUFFER_> struct FCfg {
+    static constexpr int WARPS_M = WARPS_M_, WARPS_N = WARPS_N_, MT = MT_, NT = NT_, STAGES = STAGES_, CTAS = CTAS_;
+    static constexpr int BK = BK_;
+    static constexpr bool DOUBLE_BUFFER = DOUBLE_BUFFER_;   // operand fragments of the next 4-deep step fetched before this step's DMMAs
+    static constexpr int TM = WARPS_M * MT * 8, TN = WARPS_N * NT * 8, THREADS = WARPS_M * WARPS_N * 32;
+    static constexpr int AS = BK + 4, BS = TN + 4;          // padded rows: conflict-free 8-byte fragment loads
+    static constexpr int A_Q = TM * AS, B_Q = BK * BS;      // words of one quadrant's slab
+    static constexpr int STAGE_WORDS = 4 * A_Q + 4 * B_Q;
+    static constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * sizeof(double);
+    // loader: a thread copies the 16-byte chunk (row, kc) of A and (krow, nc) of B in each of the four quadrants,
+    // and the same chunk A_ROWS_STEP / B_ROWS_STEP rows further down, A_PASSES / B_PASSES times
+    static constexpr int A_ROWS_STEP = THREADS / (BK / 2), A_PASSES = TM / A_ROWS_STEP;
+    static constexpr int B_ROWS_STEP = THREADS / (TN / 2), B_PASSES = BK / B_ROWS_STEP;
+    static_assert(A_ROWS_STEP * A_PASSES == TM && B_ROWS_STEP * B_PASSES == BK && A_PASSES >= 1 && B_PASSES >= 1,
+                  "the loader covers the slab exactly");
+    static_assert(AS % 8 == 4 && BS % 16 == 4 && STAGES >= 2, "fragment loads rely on these strides");
+};
+// 4 warps of 8 x 16 positions: tile 16 x 32.  h = 256 gives 128 CTAs, one warp per SM sub-partition, so each warp
+// hides its own shared-memory latency (fragments double-buffered in registers); two CTAs fit an SM when there are more tiles.
+#ifndef FSMALL_BK
+#define FSMALL_BK 16
+#define FSMALL_STAGES 3
+#endif
+using FSmall = FCfg<2, 2, 1, 2, FSMALL_BK, FSMALL_STAGES, 2, true>;
+// 8 warps of 16 x 16 positions: tile 32 x 64, for parents with enough tiles to fill the SMs several times.
+using FWide = FCfg<2, 4, 2, 2, 16, 3, 1, false>;
+
+__device__ __forceinline__ void cpa16(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cpa16_full(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cpa8(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cpa_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cpa_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+// D += A.B, one warp-wide 8x8x4 FP64 tensor-core operation.  g = lane / 4, q = lane % 4:
+// a = A[g][q], b = B[q][g], d0, d1 = D[g][2q], D[g][2q + 1].
+__device__ __forceinline__ void dmma1(double &d0, double &d1, double a, double b)
+{
+    asm("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
+        : "+d"(d0), "+d"(d1)
+        : "d"(a), "d"(b));
+}
+
+template <class F>
+__global__ void __launch_bounds__(F::THREADS, F::CTAS)
+fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item0, int peel)
+{
+    constexpr int TM = F::TM, TN = F::TN, BK = F::BK, AS = F::AS, BS = F::BS, A_Q = F::A_Q, B_Q = F::B_Q;
+    constexpr int MT = F::MT, NT = F::NT, STAGES = F::STAGES, STAGE_WORDS = F::STAGE_WORDS, KS = BK / 4;
+    extern __shared__ __align__(16) double smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int wm = warp / F::WARPS_N, wn = warp % F::WARPS_N;
+    const int g = lane >> 2, q = lane & 3;
+    const uint32_t smem_base = uint32_t(__cvta_generic_to_shared(smem));
+
+    const Node nd = parents[item0 + blockIdx.z];
+    const double *A = base_ptr(bases, nd.a.base) + nd.a.off;
+    const double *B = base_ptr(bases, nd.b.base) + nd.b.off;
+    const long long lda = nd.a.ld, ldb = nd.b.ld;
+    const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+    // 16-byte copies need every quadrant row to start on a 16-byte boundary
+    const bool a16 = ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && ((lda & 1) == 0) && ((h & 1) == 0);
+    const bool b16 = ((reinterpret_cast<uintptr_t>(B) & 15) == 0) && ((ldb & 1) == 0) && ((h & 1) == 0);
+    const bool interior = a16 && b16 && m0 + TM <= h && n0 + TN <= h;
+    const double *safe = reinterpret_cast<const double *>(parents);     // valid, 16-byte aligned: for copies of 0 bytes
+    const int ktiles = (h + BK - 1) / BK;
+
+    // loader coordinates and the element offsets of the four quadrants X11, X12, X21, X22
+    const int a_row = tid / (BK / 2), a_kc = tid % (BK / 2);
+    const int b_krow = tid / (TN / 2), b_nc = tid % (TN / 2);
+    const long long aq[4] = {0, h, (long long)h * lda, (long long)h * lda + h};
+    const long long bq[4] = {0, h, (long long)h * ldb, (long long)h * ldb + h};
+    const double *pa = A + (long long)(m0 + a_row) * lda + 2 * a_kc;     // advances by BK per slab
+    const double *pb = B + (long long)b_krow * ldb + n0 + 2 * b_nc;      // advances by BK rows per slab
+    const uint32_t a_dst0 = smem_base + uint32_t((a_row * AS + 2 * a_kc) * 8);
+    const uint32_t b_dst0 = smem_base + uint32_t((4 * A_Q + b_krow * BS + 2 * b_nc) * 8);
+    int load_kt = 0;
+
+    auto issue_load = [&]() {
+        if (load_kt < ktiles) {
+            const uint32_t soff = uint32_t((load_kt % STAGES) * STAGE_WORDS * 8);
+            const int k0 = load_kt * BK;
+            if (interior && k0 + BK <= h) {
+#pragma unroll
+                for (int p = 0; p < F::A_PASSES; ++p)
+#pragma unroll
+                    for (int x = 0; x < 4; ++x)
+                        cpa16_full(a_dst0 + soff + uint32_t((x * A_Q + p * F::A_ROWS_STEP * AS) * 8),
+                                   pa + aq[x] + (long long)(p * F::A_ROWS_STEP) * lda);
+#pragma unroll
+                for (int p = 0; p < F::B_PASSES; ++p)
+#pragma unroll
+                    for (int x = 0; x < 4; ++x)
+                        cpa16_full(b_dst0 + soff + uint32_t((x * B_Q + p * F::B_ROWS_STEP * BS) * 8),
+                                   pb + bq[x] + (long long)(p * F::B_ROWS_STEP) * ldb);
+            } else {
+                const int kvalid = max(0, min(2, h - (k0 + 2 * a_kc)));
+#pragma unroll
+                for (int p = 0; p < F::A_PASSES; ++p) {
+                    const int nv = (m0 + a_row + p * F::A_ROWS_STEP < h) ? kvalid : 0;
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const double *s = pa + aq[x] + (long long)(p * F::A_ROWS_STEP) * lda;
+                        const uint32_t dst = a_dst0 + soff + uint32_t((x * A_Q + p * F::A_ROWS_STEP * AS) * 8);
+                        if (a16) {
+                            cpa16(dst, nv ? s : safe, nv * 8);
+                        } else {
+                            cpa8(dst, nv >= 1 ? s : safe, nv >= 1 ? 8 : 0);
+                            cpa8(dst + 8, nv >= 2 ? s + 1 : safe, nv >= 2 ? 8 : 0);
+                        }
+                    }
+                }
+                const int cvalid = max(0, min(2, h - (n0 + 2 * b_nc)));
+#pragma unroll
+                for (int p = 0; p < F::B_PASSES; ++p) {
+                    const int nv = (k0 + b_krow + p * F::B_ROWS_STEP < h) ? cvalid : 0;
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const double *s = pb + bq[x] + (long long)(p * F::B_ROWS_STEP) * ldb;
+                        const uint32_t dst = b_dst0 + soff + uint32_t((x * B_Q + p * F::B_ROWS_STEP * BS) * 8);
+                        if (b16) {
+                            cpa16(dst, nv ? s : safe, nv * 8);
+                        } else {
+                            cpa8(dst, nv >= 1 ? s : safe, nv >= 1 ? 8 : 0);
+                            cpa8(dst + 8, nv >= 2 ? s + 1 : safe, nv >= 2 ? 8 : 0);
+                        }
+                    }
+                }
+            }
+            pa += BK;
+            pb += (long long)BK * ldb;
+            ++load_kt;
+        }
+        cpa_commit();
+    };
+
+    double acc[7][MT][NT][2];
+#pragma unroll
+    for (int j = 0; j < 7; ++j)
+#pragma unroll
+        for (int i = 0; i < MT; ++i)
+#pragma unroll
+            for (int t = 0; t < NT; ++t) acc[j][i][t][0] = acc[j][i][t][1] = 0.0;
+
+    // The seven operand fragments of one 4-deep step on each side, formed in registers from the four quadrant fragments.
+    const double *a_frag0 = smem + (wm * MT * 8 + g) * AS + q;
+    const double *b_frag0 = smem + 4 * A_Q + q * BS + wn * NT * 8 + g;
+    auto load_frags = [&](int slot, int kk, double (&ta)[MT][7], double (&sb)[NT][7]) {
+        const double *As = a_frag0 + slot * STAGE_WORDS + kk * 4, *Bs = b_frag0 + slot * STAGE_WORDS + kk * 4 * BS;
+#pragma unroll
+        for (int i = 0; i < MT; ++i) {
+            const double *p = As + i * 8 * AS;
+            const double a11 = p[0], a12 = p[A_Q], a21 = p[2 * A_Q], a22 = p[3 * A_Q];
+            const double t2 = a21 + a22, t3 = t2 - a11;
+            ta[i][0] = a11; ta[i][1] = a12; ta[i][2] = t2; ta[i][3] = t3;
+            ta[i][4] = a11 - a21; ta[i][5] = a12 - t3; ta[i][6] = a22;
+        }
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            const double *p = Bs + t * 8;
+            const double b11 = p[0], b12 = p[B_Q], b21 = p[2 * B_Q], b22 = p[3 * B_Q];
+            const double s2 = b12 - b11, s3 = b22 - s2;
+            sb[t][0] = b11; sb[t][1] = b21; sb[t][2] = s2; sb[t][3] = s3;
+            sb[t][4] = b22 - b12; sb[t][5] = b22; sb[t][6] = s3 - b21;
+        }
+    };
+    auto mma_step = [&](const double (&ta)[MT][7], const double (&sb)[NT][7]) {
+#pragma unroll
+        for (int j = 0; j < 7; ++j)
+#pragma unroll
+            for (int i = 0; i < MT; ++i)
+#pragma unroll
+                for (int t = 0; t < NT; ++t) dmma1(acc[j][i][t][0], acc[j][i][t][1], ta[i][j], sb[t][j]);
+    };
+
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) issue_load();
+    cpa_wait<STAGES - 2>();         // slab 0 has landed
+    __syncthreads();
+
+    if (F::DOUBLE_BUFFER) {
+        // One warp per scheduler has nobody to hide its shared-memory latency behind: the fragments of the next
+        // step (of the next slab, across the barrier) are fetched and summed before this step's DMMAs are issued.
+        double ta0[MT][7], sb0[NT][7], ta1[MT][7], sb1[NT][7];
+        int slot = 0;
+        load_frags(slot, 0, ta0, sb0);
+        for (int kt = 0; kt < ktiles; ++kt) {
+#pragma unroll
+            for (int kk = 0; kk < KS; kk += 2) {
+                load_frags(slot, kk + 1, ta1, sb1);
+                mma_step(ta0, sb0);
+                if (kk == 0) issue_load();      // refills the slot every warp left at the last barrier
+                if (kk + 2 < KS) {
+                    load_frags(slot, kk + 2, ta0, sb0);
+                } else {
+                    cpa_wait<STAGES - 2>();     // this thread's copies of the next slab are complete
+                    __syncthreads();            // ... and everyone's; all reads of this slab have been issued
+                    slot = slot + 1 == STAGES ? 0 : slot + 1;
+                    load_frags(slot, 0, ta0, sb0);      // past the last slab: zeros or stale data, never used
+                }
+                mma_step(ta1, sb1);
+            }
+        }
+    } else {
+        for (int kt = 0; kt < ktiles; ++kt) {
+            if (kt > 0) {
+                cpa_wait<STAGES - 2>();
+                __syncthreads();
+            }
+            issue_load();
+#pragma unroll
+            for (int kk = 0; kk < KS; ++kk) {
+                double ta[MT][7], sb[NT][7];
+                load_frags(kt % STAGES, kk, ta, sb);
+                mma_step(ta, sb);
+            }
+        }
+    }
+    cpa_wait<0>();
+
+    // U-chain in registers, four quadrants of C out
+    double *C = base_ptr(bases, nd.c.base) + nd.c.off;
+    const long long ldc = nd.c.ld, hq = (long long)h * ldc;
+    const bool c16 = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((ldc & 1) == 0) && ((h & 1) == 0);
+    const double *acol = A + 2 * h;                              // peeled parent: A[:, 2h] and B[2h, :]
+    const double *brow = B + (long long)(2 * h) * ldb;
+#pragma unroll
+    for (int i = 0; i < MT; ++i) {
+        const int r = m0 + (wm * MT + i) * 8 + g;
+        if (r >= h) continue;
+        double a0 = 0.0, a1 = 0.0;
+        if (peel) {
+            a0 = acol[(long long)r * lda];
+            a1 = acol[(long long)(r + h) * lda];
+        }
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            const int c = n0 + (wn * NT + t) * 8 + 2 * q;
+            if (c >= h) continue;
+            double v[4][2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const double q0 = acc[0][i][t][e], q1 = acc[1][i][t][e], q2 = acc[2][i][t][e], q3 = acc[3][i][t][e];
+                const double q4 = acc[4][i][t][e], q5 = acc[5][i][t][e], q6 = acc[6][i][t][e];
+                const double u1 = q0 + q3, u2 = u1 + q4, u3 = u1 + q2;
+                v[0][e] = q0 + q1;
+                v[1][e] = u3 + q5;
+                v[2][e] = u2 - q6;
+                v[3][e] = u2 + q2;
+            }
+            const bool two = c + 1 < h;
+            if (peel) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    if (e == 1 && !two) break;
+                    const double b0 = brow[c + e], b1 = brow[c + e + h];
+                    v[0][e] = fma(a0, b0, v[0][e]);
+                    v[1][e] = fma(a0, b1, v[1][e]);
+                    v[2][e] = fma(a1, b0, v[2][e]);
+                    v[3][e] = fma(a1, b1, v[3][e]);
+                }
+            }
+            double *o = C + (long long)r * ldc + c;
+            double *dst[4] = {o, o + h, o + hq, o + hq + h};
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                if (two && c16) {
+                    *reinterpret_cast<double2 *>(dst[x]) = make_double2(v[x][0], v[x][1]);
+                } else {
+                    dst[x][0] = v[x][0];
+                    if (two) dst[x][1] = v[x][1];
+                }
+            }
+        }
+    }
+}
+
+template <class F> cudaError_t configure_one()
+{
+    return cudaFuncSetAttribute(fused_step_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(F::SMEM_BYTES));
+}
+
+template <class F>
+void launch_one(const Node *parents, const Bases &bases, int h, int64_t item0, int64_t zn, int peel, cudaStream_t stream)
+{
+    const dim3 grid(unsigned((h + F::TN - 1) / F::TN), unsigned((h + F::TM - 1) / F::TM), unsigned(zn));
+    fused_step_kernel<F><<<grid, F::THREADS, F::SMEM_BYTES, stream>>>(parents, bases, h, int(item0), peel);
+}
+
+}  // namespace
+
+cudaError_t configure_fused_step_kernels()
+{
+    cudaError_t e = configure_one<FSmall>();
+    if (e != cudaSuccess) return e;
+    return configure_one<FWide>();
+}
+
+bool fused_step_uses_wide_tiles(int64_t h, int64_t count, int sms)
+{
+    // the wide tile moves half the operand bytes per flop; it needs enough tiles to keep every SM busy
+    const int64_t wide_tiles = ((h + FWide::TM - 1) / FWide::TM) * ((h + FWide::TN - 1) / FWide::TN) * count;
+    return wide_tiles >= 2 * int64_t(sms);
+}
+
+cudaError_t launch_fused_step(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
+                              int *launched)
+{
+    const Node *parents = tab + op.parent_tab;
+    const bool wide = fused_step_uses_wide_tiles(op.h, op.count, sm_count);
+    for (int64_t item0 = 0; item0 < op.count; item0 += kMaxItemsPerLaunch) {
+        const int64_t zn = op.count - item0 < kMaxItemsPerLaunch ? op.count - item0 : kMaxItemsPerLaunch;
+        if (wide) launch_one<FWide>(parents, bases, int(op.h), item0, zn, op.peel_fused, stream);
+        else launch_one<FSmall>(parents, bases, int(op.h), item0, zn, op.peel_fused, stream);
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace strassen

@@ -125,6 +125,18 @@ inline int gemm_regions(int64_t M64, int64_t count, int sms, GemmRegion *out)
     if (wide_leaves < count) out[k++] = GemmRegion{true, 0, 0, M, M, wide_leaves, count - wide_leaves};
     return k;
 }
+// One whole BFS step in one kernel (fused_step.cu): op.count parents of size 2 op.h (+ 1 when peeled).
+cudaError_t launch_fused_step(const Node *tab, const Launch &op, const Bases &bases, int sm_count, cudaStream_t stream,
+                              int *launched);
+cudaError_t configure_fused_step_kernels();
+// The fused step replaces three launches whose base products cannot fill the SMs with large tiles: it pays while
+// the children's 128 x 128 tiles number fewer than the SMs (measured on B200).
+inline bool fused_step_pays(int64_t h, int64_t parents, int sms)
+{
+    const int64_t tiles = ((h + 127) / 128) * ((h + 127) / 128) * 7 * parents;
+    return tiles < sms;
+}
+
 constexpr int kNominalSMs = 148;   // B200; used where launches are counted without a device at hand
 
 // Sets the shared-memory attribute of every GEMM kernel shape on the current device (idempotent).

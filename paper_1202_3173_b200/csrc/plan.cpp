@@ -74,7 +74,18 @@ struct Builder {
         return kids;
     }
 
-    int group_size(int level) const { return fused_group_size(p->sizes, p->schedule, level, p->max_fused_levels); }
+    // the deepest level as one fused kernel takes no part in the multi-level passes above it
+    bool fused_last() const
+    {
+        if (p->levels.empty()) return false;
+        const LevelInfo &lv = p->levels.back();
+        return fused_step_chosen(p->fused_step, p->schedule, lv.h, lv.parents);
+    }
+    int group_size(int level) const
+    {
+        const std::string sched = fused_last() ? p->schedule.substr(0, p->schedule.size() - 1) : p->schedule;
+        return fused_group_size(p->sizes, sched, level, p->max_fused_levels);
+    }
 
     // nodes of `level` are p->nodes[tab .. tab + count)
     void build(int level, int64_t tab, int64_t count)
@@ -96,7 +107,13 @@ struct Builder {
             const Node &nd = p->nodes[tab + q];
             parents_even = parents_even && even(nd.a) && even(nd.b) && even(nd.c);
         }
-        if (lv.mode == 'B') {
+        if (lv.mode == 'B' && level == L - 1 && fused_last()) {
+            Launch f{};
+            f.kind = OP_FUSED_STEP; f.level = level; f.j = -1; f.vec_ok = parents_even;
+            f.parent_tab = tab; f.child_tab = -1; f.grand_tab = -1; f.count = N; f.m = lv.m; f.h = h;
+            f.peel_fused = lv.peel;
+            p->launches.push_back(f);
+        } else if (lv.mode == 'B') {
             const int64_t ctab = append(bfs_children(tab, N, lv));
             if (ctab < 0) return;
             Launch f{};
@@ -199,39 +216,69 @@ int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched
     return run % max_fused == 0 ? max_fused : run % max_fused;
 }
 
-// Estimate of one product's time from the quantities the kernels are bound by (measured on B200): the base
-// products at the DMMA rate of their tiling, everything else as HBM bytes, a few microseconds per launch.
-// Only used to decide which candidates are tried first; the choice itself is by measurement.
-double plan_model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch)
+bool fused_step_chosen(int mode, const std::string &sched, int64_t h, int64_t parents)
+{
+    if (sched.empty() || sched.back() != 'B' || mode == 2 || h < 1) return false;
+    return mode == 1 || fused_step_pays(h, parents, kNominalSMs);
+}
+
+// What one product costs, from the quantities the kernels are bound by (measured on B200): the base products at
+// the DMMA rate of their tiling, everything else as HBM bytes, a few microseconds per launch.
+ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch, int fused_mode)
 {
     const int L = int(sched.size());
-    const double hbm = 6.2e12, launch_us = 3.0;
-    double bytes = 0.0, launches = 0.0, visits = double(batch), sequential = 1.0;   // node visits at the current level
+    ModelParts out{};
+    double visits = double(batch), sequential = 1.0;   // node visits at the current level; sub-trees run one after another
+    int64_t parents_exact = batch;
+    const bool fused = L > 0 && fused_step_chosen(fused_mode, sched, sizes[L], [&] {
+        int64_t live = batch;
+        for (int i = 0; i + 1 < L; ++i)
+            if (sched[i] == 'B') live *= 7;
+        return live;
+    }());
+    const std::string upper = fused ? sched.substr(0, size_t(L) - 1) : sched;    // levels handled by streaming passes
+    const int LU = int(upper.size());
     for (int level = 0; level < L;) {
         const double m = double(sizes[level]), h = double(sizes[level + 1]);
         if (sizes[level] & 1) {
-            bytes += visits * 2.0 * m * m * 8.0;      // last column and last row: each reads one operand in full
-            launches += 2.0 * sequential;
+            out.pass_bytes += visits * 2.0 * m * m * 8.0;      // last column and last row: each reads one operand in full
+            out.launches += 2.0 * sequential;
         }
+        if (level >= LU) break;                                // the fused deepest step: accounted with the products
         if (sched[level] == 'D') {
-            bytes += visits * 57.0 * h * h * 8.0;     // 30 h^2 to form the operands one at a time, 27 h^2 to fold the products
-            launches += 12.0 * sequential;
+            out.pass_bytes += visits * 57.0 * h * h * 8.0;     // 30 h^2 to form the operands one at a time, 27 h^2 to fold the products
+            out.launches += 12.0 * sequential;
             visits *= 7.0;
             sequential *= 7.0;
             ++level;
             continue;
         }
-        const int g = fused_group_size(sizes, sched, level, 3);
+        const int g = fused_group_size(sizes, upper, level, 3);
         const double words = g == 1 ? 27.0 : g == 2 ? 28.0 + 16.25 : 49.0 + 25.5;    // per parent, in h^2 of its children
-        bytes += visits * words * h * h * 8.0;
-        launches += 2.0 * sequential;
-        for (int i = 0; i < g; ++i) visits *= 7.0;
+        out.pass_bytes += visits * words * h * h * 8.0;
+        out.launches += 2.0 * sequential;
+        for (int i = 0; i < g; ++i) {
+            visits *= 7.0;
+            parents_exact *= 7;
+        }
         level += g;
+    }
+    if (fused) {
+        // one kernel for the whole deepest step: tiles of 16 x 32 positions, h / 16 slabs each; 0.84 us per slab for a
+        // CTA alone on its SM, 1.25 us when two share one (measured at h = 256, 384, 512)
+        const double h = double(sizes[L]);
+        const double tiles = double((sizes[L] + 15) / 16) * double((sizes[L] + 31) / 32) * visits / sequential;
+        const double slabs = double((sizes[L] + 15) / 16);
+        const double per_launch = tiles <= kNominalSMs ? slabs * 0.84 : double(int64_t((tiles + 2 * kNominalSMs - 1) / (2 * kNominalSMs))) * slabs * 1.25;
+        out.product_us += per_launch * sequential;
+        out.product_flops += visits * 7.0 * 2.0 * h * h * h;
+        out.launches += sequential;
+        return out;
     }
     const int64_t b = sizes[L];
     const double leaves = visits, kp = double((b + 15) / 16 * 16);
     const int rem = gemm_thin_remainder(b);
-    double us = 0.0;
+    out.product_flops = leaves * 2.0 * double(b) * double(b) * double(b);
     if (b - rem > 0) {
         GemmRegion regions[4];
         const int64_t count = leaves > 4.0e9 ? int64_t(4e9) : int64_t(leaves);
@@ -245,20 +292,30 @@ double plan_model_ms(const std::vector<int64_t> &sizes, const std::string &sched
             const double tile_us = r.small ? wide_tile_us * 0.5 / 0.88 : wide_tile_us;
             double rounds = tiles / sequential / slots;          // per launch: a DFS level above runs its sub-trees one by one
             if (rounds < 1.0) rounds = 1.0;
-            us += rounds * tile_us * sequential;
-            launches += sequential;
+            out.product_us += rounds * tile_us * sequential;
+            out.launches += sequential;
         }
     }
     if (rem) {
-        bytes += leaves * 2.0 * double(b) * double(b) * 8.0;
-        launches += 2.0 * sequential;
+        out.thin_bytes += leaves * 2.0 * double(b) * double(b) * 8.0;
+        out.launches += 2.0 * sequential;
     }
-    return us * 1e-3 + bytes / hbm * 1e3 + launches * launch_us * 1e-3;
+    (void)parents_exact;
+    return out;
+}
+
+// Only used to decide which candidates are tried first and to pick plans created with cutoff 0; the autotuner's
+// choice itself is by measurement.
+double plan_model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch, int fused_mode)
+{
+    const double hbm = 6.2e12, launch_us = 3.0;
+    const ModelParts m = plan_model_parts(sizes, sched, batch, fused_mode);
+    return m.product_us * 1e-3 + (m.pass_bytes + m.thin_bytes) / hbm * 1e3 + m.launches * launch_us * 1e-3;
 }
 
 
-bool model_choice(int64_t n, int64_t batch, int64_t budget_words, int64_t min_base, std::vector<int64_t> *sizes_out,
-                  std::string *sched_out)
+bool model_choice(int64_t n, int64_t batch, int64_t budget_words, int64_t min_base, int fused_mode,
+                  std::vector<int64_t> *sizes_out, std::string *sched_out)
 {
     std::vector<int64_t> chain{n};
     while (chain.back() / 2 >= min_base && chain.size() <= 10) chain.push_back(chain.back() / 2);
@@ -274,7 +331,7 @@ bool model_choice(int64_t n, int64_t batch, int64_t budget_words, int64_t min_ba
             double nodes = double(batch), level_nodes = double(batch);      // entries the node tables would need
             for (size_t i = 0; i < L; ++i) nodes += (level_nodes *= 7.0);
             if (nodes > double(kMaxNodes)) continue;
-            const double ms = plan_model_ms(sizes, sched, batch);
+            const double ms = plan_model_ms(sizes, sched, batch, fused_mode);
             if (best < 0 || ms < best) {
                 best = ms;
                 *sizes_out = sizes;

@@ -38,7 +38,8 @@ enum OpKind : int32_t {
     OP_SCALE_IN = 8,   // diagonal scaling: exponents, scaled copies of A and B in the workspace
     OP_SCALE_OUT = 9,  // diagonal scaling: C scaled back in place
     OP_FORM3 = 10,     // three BFS levels at once: sums of the children, grandchildren and great-grandchildren
-    OP_RECOMBINE3 = 11 // three BFS levels at once: 343 great-grandchild products -> the parent's C
+    OP_RECOMBINE3 = 11, // three BFS levels at once: 343 great-grandchild products -> the parent's C
+    OP_FUSED_STEP = 12  // a whole BFS step of the deepest level in one kernel: quadrants of A, B -> C
 };
 
 // Regular layout of the workspace regions a two- or three-level launch writes / reads (element offsets
@@ -92,6 +93,7 @@ struct PlanDesc {
     int64_t lda = 0, ldb = 0, ldc = 0;
     int64_t stride_a = 0, stride_b = 0, stride_c = 0;
     int max_fused_levels = 3;       // consecutive BFS levels formed / recombined by one pass: up to 3, 2 or 1
+    int fused_step = 0;             // deepest BFS step as one kernel: 0 = where the rule says it pays, 1 = always, 2 = never
     bool scale_inside = false, scale_outside = false;   // diagonal scaling (Section 6.1)
     int64_t scale_a_off = 0, scale_b_off = 0, scale_exp_off = 0, scale_ld = 0;   // workspace words / leading dimension
     std::string schedule;           // resolved, one char per level
@@ -106,15 +108,26 @@ struct PlanDesc {
 // `sched` with level sizes `sizes`; 1 for a DFS level.
 int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused);
 
+// Whether the deepest level (a BFS step over `parents` nodes with children of size h) runs as one fused kernel.
+bool fused_step_chosen(int mode, const std::string &sched, int64_t h, int64_t parents);
+
 // Cost-model estimate (milliseconds on a B200) of one product with level sizes `sizes` (m_0 .. m_L) and
 // schedule `sched`; orders the autotuner's search and picks plans created with cutoff 0.
-double plan_model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch);
+double plan_model_ms(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch, int fused_mode = 0);
+
+// The parts of that estimate, also reported as the plan's algorithmic work: bytes the streaming passes move as
+// scheduled (multi-level passes counted with what they really read and write; DFS steps with their surcharge;
+// peeled columns and rows), bytes of the thin remainder products, time and flops of the base products, launches.
+struct ModelParts {
+    double pass_bytes, thin_bytes, product_us, product_flops, launches;
+};
+ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string &sched, int64_t batch, int fused_mode = 0);
 
 // The (level sizes, schedule) of least estimated time among all step counts whose base size is >= min_base
 // and all B/D strings whose workspace fits budget_words.  False if nothing fits (cannot happen: zero levels
 // need no workspace).
-bool model_choice(int64_t n, int64_t batch, int64_t budget_words, int64_t min_base, std::vector<int64_t> *sizes_out,
-                  std::string *sched_out);
+bool model_choice(int64_t n, int64_t batch, int64_t budget_words, int64_t min_base, int fused_mode,
+                  std::vector<int64_t> *sizes_out, std::string *sched_out);
 
 // Level sizes m_0 = n, m_{i+1} = floor(m_i / 2) while m_i > cutoff.
 std::vector<int64_t> level_sizes(int64_t n, int64_t cutoff);

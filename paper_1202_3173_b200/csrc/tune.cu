@@ -69,7 +69,7 @@ extern "C" int strassen_autotune(const strassen_tune_request *req, strassen_tune
                 if (mask >> i & 1) sched[i] = 'D';
             const int64_t words = actual_workspace_words(chain, sched, batch);
             if (words < 0 || size_t(words) > req->workspace_bytes / 8) continue;       // does not fit the workspace
-            candidates.push_back(Candidate{sizes[L], sched, plan_model_ms(chain, sched, batch)});
+            candidates.push_back(Candidate{sizes[L], sched, plan_model_ms(chain, sched, batch, 0)});
         }
     }
     // most promising first, so that a search cut short by max_seconds has seen the likely winners

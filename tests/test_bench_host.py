@@ -77,3 +77,20 @@ def test_reference_arm_prints_the_contract_line():
     assert line["impl"] == "reference" and line["unit"] == "GFLOP/s" and line["higher_is_better"] is True
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"] > 0
+
+
+def test_gpus_n_without_a_launcher_starts_n_ranks():
+    """`python bench.py --gpus 2` started plainly must become two ranks by itself; the stand-in mode runs the same
+    launch path and the same max-over-ranks reduction over gloo, with no GPU work."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.check_output([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--check-launch"],
+                                  cwd=ROOT, text=True, timeout=300, env=env, stderr=subprocess.DEVNULL)
+    line = json.loads([l for l in out.strip().splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak"
+    assert line["ms_per_step"] == 4.0                                    # the slower of the ranks' 3 and 4 ms
+    assert line["value"] == pytest.approx(2 * 2 * 4096 ** 3 / 4.0e-3 / 1e9)
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.self_launch_command(8, ["--gpus", "8", "--steps", "5"])
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node" in cmd and cmd[cmd.index("--nproc-per-node") + 1] == "8"
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-4:] == ["--gpus", "8", "--steps", "5"]

@@ -231,6 +231,58 @@ def test_batch_with_two_level_passes():
     check_full(260, 65, "BB", "int8", 122, batch=3)      # odd quarter size: 8-byte accesses
 
 
+# ---- the deepest BFS step as one fused kernel ------------------------------------------------
+
+FUSED, UNFUSED = binding.STRASSEN_FLAG_FUSED_STEP, binding.STRASSEN_FLAG_NO_FUSED_STEP
+
+
+@pytest.mark.parametrize("n,cutoff,sched,batch,dist", [
+    (512, 256, "B", 1, "uniform"), (512, 256, "B", 1, "int8"),      # the small configuration: 128 CTAs of the small tile
+    (64, 32, "B", 1, "int8"), (2, 1, "B", 3, "int8"), (6, 3, "B", 1, "int8"),
+    (100, 50, "B", 2, "normal"),        # ragged tiles in both directions, inner dimension not a multiple of 16
+    (101, 50, "B", 2, "int8"),          # odd parent: rank-one term inside the kernel, then the peeled column and row
+    (258, 129, "B", 1, "int8"),         # odd quadrant size: 8-byte copies only
+    (1024, 512, "B", 1, "uniform"),     # the wide tile
+    (1030, 515, "B", 1, "int8"), (777, 388, "B", 1, "uniform"),
+    (1024, 128, "BBB", 1, "uniform"),   # two-level pass above a fused deepest step
+    (1000, 125, "DBB", 1, "int8"), (520, 65, "BDB", 2, "int8"), (771, 96, "BBB", 1, "int8"),
+    (4096, 512, "BBB", 1, "uniform"),
+])
+def test_fused_step_gives_the_bits_of_the_three_launch_path(n, cutoff, sched, batch, dist):
+    A, B = inputs.pair(n, dist, 40 + n, device="cuda", batch=None if batch == 1 else batch)
+    fused = run_plan(n, cutoff, sched, A, B, batch=batch, flags=FUSED)
+    plain = run_plan(n, cutoff, sched, A, B, batch=batch, flags=UNFUSED)
+    base = oracle.level_sizes(n, cutoff)[-1]
+    if dist == "int8" or not 1 <= base % 64 <= 8:
+        assert torch.equal(fused, plain)             # same operations in the same order on every element
+    else:       # the three-launch path sums the last 1..8 rows / columns of such a base product in another order
+        assert float((fused - plain).abs().max()) <= 1e-3 * bound(n, A, B)
+    p = Plan(n, cutoff, sched, batch=batch, flags=FUSED)
+    assert p.launches_by_kind()["fused_step"] >= 1 and p.launches_by_kind()["gemm"] == 0
+    p.close()
+    if n <= 2100:
+        check_full(n, cutoff, sched, dist, 40 + n, batch=batch, flags=FUSED)
+    else:
+        check_sampled(n, cutoff, sched, dist, 40 + n, batch=batch, flags=FUSED)
+
+
+def test_fused_step_on_pointers_that_are_only_8_byte_aligned_and_strided_views():
+    n, ld = 130, 137
+    g = torch.Generator("cuda").manual_seed(9)
+    Abuf = torch.randint(-8, 9, (n * ld + 1,), device="cuda", generator=g).double()
+    Bbuf = torch.randint(-8, 9, (n * ld + 1,), device="cuda", generator=g).double()
+    Cbuf = torch.full((n * ld + 1,), 55.0, device="cuda", dtype=torch.float64)
+    A, B, C = (x[1:].view(n, ld) for x in (Abuf, Bbuf, Cbuf))
+    plan = Plan(n, 65, "B", lda=ld, ldb=ld, ldc=ld, flags=FUSED)
+    assert plan.launches_by_kind()["fused_step"] == 1
+    binding.strassen_dgemm(plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    plan.close()
+    ref = oracle.classical(A[:, :n].cpu().numpy().copy(), B[:, :n].cpu().numpy().copy())
+    assert np.array_equal(C[:, :n].cpu().numpy(), ref)
+    assert bool((C[:, n:] == 55.0).all()) and float(Cbuf[0]) == 55.0
+
+
 def test_cuda_graph_replay_matches_launch_by_launch():
     n = 512
     A, B = inputs.pair(n, "uniform", 131, device="cuda")
