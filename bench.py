@@ -227,22 +227,29 @@ def absmax(X):
     return max(abs(float(lo)), abs(float(hi)))
 
 
-def timed_steps(fn, steps, stream, barrier=None):
-    """K steps in one timed region with a CUDA event between consecutive steps (no host synchronisation inside):
-    returns the per-step intervals in ms and the wall-clock bracket of the region."""
+def timed_steps(fn, steps, stream, barrier=None, stride=1):
+    """K steps in one timed region with a CUDA event after every `stride` steps (no host synchronisation inside):
+    returns the per-step times of the intervals in ms, the mean over the whole region, and its wall-clock bracket.
+    A stride above 1 is for steps of a few microseconds, where an event after each would be a good part of it."""
     import torch
-    events = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    marks = list(range(stride, steps, stride)) + [steps]
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(len(marks) + 1)]
     w0 = time.time()
     events[0].record(stream)
+    k = 0
     for i in range(steps):
         fn()
-        events[i + 1].record(stream)
+        if i + 1 == marks[k]:
+            k += 1
+            events[k].record(stream)
     if barrier:
         barrier()
     else:
         torch.cuda.synchronize()
     w1 = time.time()
-    return [events[i].elapsed_time(events[i + 1]) for i in range(steps)], events[0].elapsed_time(events[steps]) / steps, w0, w1
+    spans = [marks[0]] + [marks[i] - marks[i - 1] for i in range(1, len(marks))]
+    per_step = [events[i].elapsed_time(events[i + 1]) / spans[i] for i in range(len(marks))]
+    return per_step, events[0].elapsed_time(events[-1]) / steps, w0, w1
 
 
 def measure(name, steps, warmup, rank, world, dev, sampler_factory=None, want_cublas=True, want_oracle=True):
@@ -269,8 +276,14 @@ def measure(name, steps, warmup, rank, world, dev, sampler_factory=None, want_cu
     for _ in range(warmup):
         plan(A, B, out=C)
     barrier()
+    # steps of a few microseconds: one event per ~20 steps instead of one per step
+    t0 = time.perf_counter()
+    for _ in range(3):
+        plan(A, B, out=C)
+    torch.cuda.synchronize()
+    stride = 1 if (time.perf_counter() - t0) / 3 > 200e-6 else max(1, min(20, steps // 10))
     sampler = sampler_factory() if sampler_factory else None
-    per_step, ms_mean_local, w0, w1 = timed_steps(lambda: plan(A, B, out=C), steps, stream, barrier)
+    per_step, ms_mean_local, w0, w1 = timed_steps(lambda: plan(A, B, out=C), steps, stream, barrier, stride)
     clocks = sampler.stop(w0, w1) if sampler else None
     ms_median_local = statistics.median(per_step)
     ms = reduce_max(ms_median_local, dev)
@@ -293,7 +306,7 @@ def measure(name, steps, warmup, rank, world, dev, sampler_factory=None, want_cu
     add_ms = sum(v for k, v in kinds.items() if k not in ("gemm", "fused_step", "scale"))
     out = {
         "workload": name, "n": n, "batch": batch, "schedule": plan.schedule, "levels": sizes,
-        "workspace_bytes": plan.workspace_bytes, "steps": steps, "launches_per_step": plan.launch_count,
+        "workspace_bytes": plan.workspace_bytes, "steps": steps, "steps_per_event": stride, "launches_per_step": plan.launch_count,
         "launches_by_kind": {k: v for k, v in plan.launches_by_kind().items() if v},
         "ms_per_step": ms, "ms_per_step_mean": ms_mean, "ms_per_step_min": min(per_step), "ms_per_step_max": max(per_step),
         "effective_gflops": whole_job_value(n, batch, ms, 1),
@@ -326,12 +339,12 @@ def measure(name, steps, warmup, rank, world, dev, sampler_factory=None, want_cu
 
     if want_cublas:
         Cc = C if 3 * batch * n * n * 8 > 40e9 else torch.empty_like(A)      # no room for a fourth matrix at the largest size
-        reps = max(2, min(steps, 20 if n <= 4096 else 5))
+        reps = max(2, min(steps, 200 if n <= 512 else 20 if n <= 4096 else 5))
         try:
             for _ in range(3 if n <= 16384 else 1):
                 torch.matmul(A, B, out=Cc)
             torch.cuda.synchronize()
-            c_steps, c_mean, _, _ = timed_steps(lambda: torch.matmul(A, B, out=Cc), reps, stream)     # same protocol as ours
+            c_steps, c_mean, _, _ = timed_steps(lambda: torch.matmul(A, B, out=Cc), reps, stream, None, stride)     # same protocol as ours
             cms = statistics.median(c_steps)
             out["cublas_dgemm"] = {"ms": cms, "ms_mean": c_mean, "steps": reps, "gflops": 2.0 * n ** 3 * batch / (cms * 1e-3) / 1e9}
             out["vs_cublas"] = cms / ms_median_local
@@ -632,8 +645,8 @@ def main():
     line = {
         "metric": METRIC, "value": ours_gflops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "ms_per_step_mean": head["ms_per_step_mean"],
-        "timing": "median of the %d per-step CUDA-event intervals of one timed region (barrier + synchronize on both sides, "
-                  "no per-launch events inside); max over ranks" % args.steps,
+        "timing": "median over the CUDA-event intervals (one event per %d step(s)) of one timed region of %d steps (barrier + "
+                  "synchronize on both sides, no per-launch events inside); max over ranks" % (head["steps_per_event"], args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
         "config": {"workload": describe(args.workload), "schedule": sched_resolved, "levels": head["levels"],

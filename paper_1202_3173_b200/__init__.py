@@ -29,6 +29,7 @@ class Plan:
                                                   stride_c, workspace_budget_bytes, flags)
         self._ws = None
         self._packed = not (lda or ldb or ldc or stride_a or stride_b or stride_c)
+        self._want = (self.n, self.n) if self.batch == 1 else (self.batch, self.n, self.n)
 
     # -- introspection -------------------------------------------------------------
     @property
@@ -96,18 +97,19 @@ class Plan:
             raise ValueError("the plan has been closed")
         if not self._packed:
             raise ValueError("plans with leading dimensions or strides take raw pointers (binding.strassen_dgemm)")
-        want = (self.n, self.n) if self.batch == 1 else (self.batch, self.n, self.n)
+        want, f64, dev0 = self._want, torch.float64, tensors[0].device
         for name, t in zip(what, tensors):
-            if t.dtype != torch.float64:
+            if t.shape == want and t.dtype is f64 and t.is_cuda is cuda and t.is_contiguous() and t.device == dev0:
+                continue
+            if t.dtype != f64:
                 raise ValueError("%s must be float64, not %s" % (name, t.dtype))
-            if tuple(t.shape) != want and not (self.batch == 1 and tuple(t.shape) == (1,) + want):
+            if tuple(t.shape) != want:
                 raise ValueError("%s has shape %s; the plan is for %s" % (name, tuple(t.shape), want))
             if not t.is_contiguous():
                 raise ValueError("%s must be contiguous" % name)
             if t.is_cuda != cuda:
                 raise ValueError("%s must be a %s tensor" % (name, "CUDA" if cuda else "host"))
-            if cuda and t.device != tensors[0].device:
-                raise ValueError("%s is on %s, A on %s" % (name, t.device, tensors[0].device))
+            raise ValueError("%s is on %s, A on %s" % (name, t.device, dev0))
 
     def __call__(self, A, B, out=None):
         """C = A @ B for CUDA float64 tensors of the plan's shape, enqueued on the current stream."""
@@ -117,10 +119,15 @@ class Plan:
             out = torch.empty_like(A)
         else:
             self._check(("A", "B", "out"), True, A, B, out)
-        self._ensure_workspace(A.device)
-        with torch.cuda.device(A.device):
-            stream = torch.cuda.current_stream().cuda_stream
-            binding.strassen_dgemm(self._h, A.data_ptr(), B.data_ptr(), out.data_ptr(), stream)
+        if self._ws is None:
+            self._ensure_workspace(A.device)
+        index = A.device.index
+        if index == torch.cuda.current_device():
+            binding.strassen_dgemm(self._h, A.data_ptr(), B.data_ptr(), out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        else:
+            with torch.cuda.device(index):
+                binding.strassen_dgemm(self._h, A.data_ptr(), B.data_ptr(), out.data_ptr(),
+                                       torch.cuda.current_stream().cuda_stream)
         return out
 
     def run_host(self, A, B, out):

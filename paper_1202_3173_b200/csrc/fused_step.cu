@@ -16,7 +16,9 @@
 //     C12 = U3 + Q5, C21 = U2 - Q6, C22 = U2 + Q2) in registers and stores the four quadrants of C,
 //     with the rank-one term of a peeled (odd-size) parent added on the way out.
 // The operations on every element are those of the three-launch path (formation, base products,
-// recombination) in the same order, so the results have the same bits.
+// recombination); with one warp per tile they also come in the same order and the results have the
+// same bits, with two warps per tile each product is the sum of two partial sums over alternate
+// 4-deep steps (deterministic, a few ulps from the other order, exact on integer data).
 //
 // What it costs: every CTA re-reads its row panel of A and column panel of B, so the operands cross
 // L2 -> SM about (h / tile) times instead of once, and the seven accumulator sets cap the warp tile
@@ -28,32 +30,42 @@ namespace strassen {
 
 namespace {
 
-template <int WARPS_M_, int WARPS_N_, int MT_, int NT_, int BK_, int STAGES_, int CTAS_, bool DOUBLE_BUFFER_> struct FCfg {
+template <int WARPS_M_, int WARPS_N_, int KSPLIT_, int MT_, int NT_, int BK_, int STAGES_, int CTAS_, bool DOUBLE_BUFFER_> struct FCfg {
     static constexpr int WARPS_M = WARPS_M_, WARPS_N = WARPS_N_, MT = MT_, NT = NT_, STAGES = STAGES_, CTAS = CTAS_;
     static constexpr int BK = BK_;
     static constexpr bool DOUBLE_BUFFER = DOUBLE_BUFFER_;   // operand fragments of the next 4-deep step fetched before this step's DMMAs
-    static constexpr int TM = WARPS_M * MT * 8, TN = WARPS_N * NT * 8, THREADS = WARPS_M * WARPS_N * 32;
+    // KSPLIT warps share one tile of positions and take the 4-deep steps of every slab in turn (their partial
+    // products are added through shared memory at the end): two warps per SM sub-partition where the tiles are few.
+    static constexpr int KSPLIT = KSPLIT_;
+    static constexpr int TILE_WARPS = WARPS_M * WARPS_N;
+    static constexpr int TM = WARPS_M * MT * 8, TN = WARPS_N * NT * 8, THREADS = TILE_WARPS * KSPLIT * 32;
+    static constexpr int STEPS = BK / 4 / KSPLIT;           // 4-deep steps of a slab per warp
     static constexpr int AS = BK + 4, BS = TN + 4;          // padded rows: conflict-free 8-byte fragment loads
     static constexpr int A_Q = TM * AS, B_Q = BK * BS;      // words of one quadrant's slab
     static constexpr int STAGE_WORDS = 4 * A_Q + 4 * B_Q;
+    static constexpr int RED_WORDS = KSPLIT > 1 ? TILE_WARPS * (KSPLIT - 1) * 7 * MT * NT * 2 * 32 : 0;
     static constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * sizeof(double);
-    // loader: a thread copies the 16-byte chunk (row, kc) of A and (krow, nc) of B in each of the four quadrants,
-    // and the same chunk A_ROWS_STEP / B_ROWS_STEP rows further down, A_PASSES / B_PASSES times
-    static constexpr int A_ROWS_STEP = THREADS / (BK / 2), A_PASSES = TM / A_ROWS_STEP;
-    static constexpr int B_ROWS_STEP = THREADS / (TN / 2), B_PASSES = BK / B_ROWS_STEP;
-    static_assert(A_ROWS_STEP * A_PASSES == TM && B_ROWS_STEP * B_PASSES == BK && A_PASSES >= 1 && B_PASSES >= 1,
+    // loader: a thread copies the 16-byte chunk at one position (row, kc) of A / (krow, nc) of B in A_QPT / B_QPT
+    // of the four quadrants, and the same chunk A_ROWS_STEP / B_ROWS_STEP rows further down, A_PASSES / B_PASSES times
+    static constexpr int A_POS = TM * (BK / 2), B_POS = BK * (TN / 2);
+    static constexpr int A_GROUPS = THREADS >= A_POS ? THREADS / A_POS : 1, A_QPT = 4 / A_GROUPS;
+    static constexpr int B_GROUPS = THREADS >= B_POS ? THREADS / B_POS : 1, B_QPT = 4 / B_GROUPS;
+    static constexpr int A_PASSES = THREADS >= A_POS ? 1 : A_POS / THREADS, A_ROWS_STEP = THREADS >= A_POS ? TM : THREADS / (BK / 2);
+    static constexpr int B_PASSES = THREADS >= B_POS ? 1 : B_POS / THREADS, B_ROWS_STEP = THREADS >= B_POS ? BK : THREADS / (TN / 2);
+    static_assert(A_GROUPS * A_QPT == 4 && B_GROUPS * B_QPT == 4 && A_PASSES * A_ROWS_STEP == TM && B_PASSES * B_ROWS_STEP == BK,
                   "the loader covers the slab exactly");
-    static_assert(AS % 8 == 4 && BS % 16 == 4 && STAGES >= 2, "fragment loads rely on these strides");
+    static_assert(A_GROUPS * A_POS * A_PASSES == (THREADS >= A_POS ? THREADS : A_POS), "every thread has a place in the A loader");
+    static_assert(AS % 8 == 4 && BS % 16 == 4 && STAGES >= 2 && STEPS >= 2 && STEPS % 2 == 0, "fragment loads rely on these strides");
+    static_assert(RED_WORDS <= STAGES * STAGE_WORDS, "the partial products fit in the ring once it has drained");
 };
-// 4 warps of 8 x 16 positions: tile 16 x 32.  h = 256 gives 128 CTAs, one warp per SM sub-partition, so each warp
-// hides its own shared-memory latency (fragments double-buffered in registers); two CTAs fit an SM when there are more tiles.
-#ifndef FSMALL_BK
-#define FSMALL_BK 16
-#define FSMALL_STAGES 3
-#endif
-using FSmall = FCfg<2, 2, 1, 2, FSMALL_BK, FSMALL_STAGES, 2, true>;
+// Tile 16 x 32 positions: 4 warp tiles of 8 x 16, each shared by two warps that alternate over the 4-deep steps.
+// h = 256 gives 128 CTAs of 8 warps: two warps per SM sub-partition, which hide each other's latencies (one alone
+// kept the tensor pipe 52 % busy: its own operand sums and shared-memory loads sit between its DMMAs).
+using FSplit = FCfg<2, 2, 2, 1, 2, 16, 3, 1, true>;
+// The same tile with one warp per warp tile: two CTAs per SM do the hiding once the tiles outnumber the SMs.
+using FSmall = FCfg<2, 2, 1, 1, 2, 16, 3, 2, true>;
 // 8 warps of 16 x 16 positions: tile 32 x 64, for parents with enough tiles to fill the SMs several times.
-using FWide = FCfg<2, 4, 2, 2, 16, 3, 1, false>;
+using FWide = FCfg<2, 4, 1, 2, 2, 16, 3, 1, false>;
 
 __device__ __forceinline__ void cpa16(uint32_t dst, const void *src, int src_bytes)
 {
@@ -84,10 +96,11 @@ __global__ void __launch_bounds__(F::THREADS, F::CTAS)
 fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item0, int peel)
 {
     constexpr int TM = F::TM, TN = F::TN, BK = F::BK, AS = F::AS, BS = F::BS, A_Q = F::A_Q, B_Q = F::B_Q;
-    constexpr int MT = F::MT, NT = F::NT, STAGES = F::STAGES, STAGE_WORDS = F::STAGE_WORDS, KS = BK / 4;
+    constexpr int MT = F::MT, NT = F::NT, STAGES = F::STAGES, STAGE_WORDS = F::STAGE_WORDS, KSPLIT = F::KSPLIT;
     extern __shared__ __align__(16) double smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int wm = warp / F::WARPS_N, wn = warp % F::WARPS_N;
+    const int tw = warp % F::TILE_WARPS, ks = warp / F::TILE_WARPS;      // warp tile; which of the 4-deep steps are mine
+    const int wm = tw / F::WARPS_N, wn = tw % F::WARPS_N;
     const int g = lane >> 2, q = lane & 3;
     const uint32_t smem_base = uint32_t(__cvta_generic_to_shared(smem));
 
@@ -104,10 +117,12 @@ fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item
     const int ktiles = (h + BK - 1) / BK;
 
     // loader coordinates and the element offsets of the four quadrants X11, X12, X21, X22
-    const int a_row = tid / (BK / 2), a_kc = tid % (BK / 2);
-    const int b_krow = tid / (TN / 2), b_nc = tid % (TN / 2);
-    const long long aq[4] = {0, h, (long long)h * lda, (long long)h * lda + h};
-    const long long bq[4] = {0, h, (long long)h * ldb, (long long)h * ldb + h};
+    const int a_pos = tid % (F::A_GROUPS > 1 ? F::A_POS : F::THREADS), a_q0 = F::A_GROUPS > 1 ? (tid / F::A_POS) * F::A_QPT : 0;
+    const int b_pos = tid % (F::B_GROUPS > 1 ? F::B_POS : F::THREADS), b_q0 = F::B_GROUPS > 1 ? (tid / F::B_POS) * F::B_QPT : 0;
+    const int a_row = a_pos / (BK / 2), a_kc = a_pos % (BK / 2);
+    const int b_krow = b_pos / (TN / 2), b_nc = b_pos % (TN / 2);
+    const auto aq = [&](int x) { return (long long)(x >> 1) * h * lda + (x & 1) * h; };
+    const auto bq = [&](int x) { return (long long)(x >> 1) * h * ldb + (x & 1) * h; };
     const double *pa = A + (long long)(m0 + a_row) * lda + 2 * a_kc;     // advances by BK per slab
     const double *pb = B + (long long)b_krow * ldb + n0 + 2 * b_nc;      // advances by BK rows per slab
     const uint32_t a_dst0 = smem_base + uint32_t((a_row * AS + 2 * a_kc) * 8);
@@ -122,23 +137,23 @@ fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item
 #pragma unroll
                 for (int p = 0; p < F::A_PASSES; ++p)
 #pragma unroll
-                    for (int x = 0; x < 4; ++x)
+                    for (int x = a_q0; x < a_q0 + F::A_QPT; ++x)
                         cpa16_full(a_dst0 + soff + uint32_t((x * A_Q + p * F::A_ROWS_STEP * AS) * 8),
-                                   pa + aq[x] + (long long)(p * F::A_ROWS_STEP) * lda);
+                                   pa + aq(x) + (long long)(p * F::A_ROWS_STEP) * lda);
 #pragma unroll
                 for (int p = 0; p < F::B_PASSES; ++p)
 #pragma unroll
-                    for (int x = 0; x < 4; ++x)
+                    for (int x = b_q0; x < b_q0 + F::B_QPT; ++x)
                         cpa16_full(b_dst0 + soff + uint32_t((x * B_Q + p * F::B_ROWS_STEP * BS) * 8),
-                                   pb + bq[x] + (long long)(p * F::B_ROWS_STEP) * ldb);
+                                   pb + bq(x) + (long long)(p * F::B_ROWS_STEP) * ldb);
             } else {
                 const int kvalid = max(0, min(2, h - (k0 + 2 * a_kc)));
 #pragma unroll
                 for (int p = 0; p < F::A_PASSES; ++p) {
                     const int nv = (m0 + a_row + p * F::A_ROWS_STEP < h) ? kvalid : 0;
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const double *s = pa + aq[x] + (long long)(p * F::A_ROWS_STEP) * lda;
+                    for (int x = a_q0; x < a_q0 + F::A_QPT; ++x) {
+                        const double *s = pa + aq(x) + (long long)(p * F::A_ROWS_STEP) * lda;
                         const uint32_t dst = a_dst0 + soff + uint32_t((x * A_Q + p * F::A_ROWS_STEP * AS) * 8);
                         if (a16) {
                             cpa16(dst, nv ? s : safe, nv * 8);
@@ -153,8 +168,8 @@ fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item
                 for (int p = 0; p < F::B_PASSES; ++p) {
                     const int nv = (k0 + b_krow + p * F::B_ROWS_STEP < h) ? cvalid : 0;
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const double *s = pb + bq[x] + (long long)(p * F::B_ROWS_STEP) * ldb;
+                    for (int x = b_q0; x < b_q0 + F::B_QPT; ++x) {
+                        const double *s = pb + bq(x) + (long long)(p * F::B_ROWS_STEP) * ldb;
                         const uint32_t dst = b_dst0 + soff + uint32_t((x * B_Q + p * F::B_ROWS_STEP * BS) * 8);
                         if (b16) {
                             cpa16(dst, nv ? s : safe, nv * 8);
@@ -217,24 +232,24 @@ fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item
     __syncthreads();
 
     if (F::DOUBLE_BUFFER) {
-        // One warp per scheduler has nobody to hide its shared-memory latency behind: the fragments of the next
-        // step (of the next slab, across the barrier) are fetched and summed before this step's DMMAs are issued.
+        // Fragments double-buffered in registers: those of the warp's next step (of the next slab, across the
+        // barrier) are fetched and summed before this step's DMMAs are issued.
         double ta0[MT][7], sb0[NT][7], ta1[MT][7], sb1[NT][7];
         int slot = 0;
-        load_frags(slot, 0, ta0, sb0);
+        load_frags(slot, ks, ta0, sb0);
         for (int kt = 0; kt < ktiles; ++kt) {
 #pragma unroll
-            for (int kk = 0; kk < KS; kk += 2) {
-                load_frags(slot, kk + 1, ta1, sb1);
+            for (int i = 0; i < F::STEPS; i += 2) {
+                load_frags(slot, ks + KSPLIT * (i + 1), ta1, sb1);
                 mma_step(ta0, sb0);
-                if (kk == 0) issue_load();      // refills the slot every warp left at the last barrier
-                if (kk + 2 < KS) {
-                    load_frags(slot, kk + 2, ta0, sb0);
+                if (i == 0) issue_load();       // refills the slot every warp left at the last barrier
+                if (i + 2 < F::STEPS) {
+                    load_frags(slot, ks + KSPLIT * (i + 2), ta0, sb0);
                 } else {
                     cpa_wait<STAGES - 2>();     // this thread's copies of the next slab are complete
                     __syncthreads();            // ... and everyone's; all reads of this slab have been issued
                     slot = slot + 1 == STAGES ? 0 : slot + 1;
-                    load_frags(slot, 0, ta0, sb0);      // past the last slab: zeros or stale data, never used
+                    load_frags(slot, ks, ta0, sb0);     // past the last slab: stale data, never used
                 }
                 mma_step(ta1, sb1);
             }
@@ -247,14 +262,44 @@ fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item
             }
             issue_load();
 #pragma unroll
-            for (int kk = 0; kk < KS; ++kk) {
+            for (int i = 0; i < F::STEPS; ++i) {
                 double ta[MT][7], sb[NT][7];
-                load_frags(kt % STAGES, kk, ta, sb);
+                load_frags(kt % STAGES, ks + KSPLIT * i, ta, sb);
                 mma_step(ta, sb);
             }
         }
     }
     cpa_wait<0>();
+    if (KSPLIT > 1) {
+        // the warps that took the later steps hand their partial products over through the drained ring
+        __syncthreads();
+        constexpr int PER_WARP = 7 * MT * NT * 2 * 32;
+        if (ks > 0) {
+            double *red = smem + ((ks - 1) * F::TILE_WARPS + tw) * PER_WARP + lane;
+#pragma unroll
+            for (int j = 0; j < 7; ++j)
+#pragma unroll
+                for (int i = 0; i < MT; ++i)
+#pragma unroll
+                    for (int t = 0; t < NT; ++t)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) red[(((j * MT + i) * NT + t) * 2 + e) * 32] = acc[j][i][t][e];
+        }
+        __syncthreads();
+        if (ks > 0) return;
+#pragma unroll
+        for (int s2 = 1; s2 < KSPLIT; ++s2) {
+            const double *red = smem + ((s2 - 1) * F::TILE_WARPS + tw) * PER_WARP + lane;
+#pragma unroll
+            for (int j = 0; j < 7; ++j)
+#pragma unroll
+                for (int i = 0; i < MT; ++i)
+#pragma unroll
+                    for (int t = 0; t < NT; ++t)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) acc[j][i][t][e] += red[(((j * MT + i) * NT + t) * 2 + e) * 32];
+        }
+    }
 
     // U-chain in registers, four quadrants of C out
     double *C = base_ptr(bases, nd.c.base) + nd.c.off;
@@ -329,9 +374,10 @@ void launch_one(const Node *parents, const Bases &bases, int h, int64_t item0, i
 
 cudaError_t configure_fused_step_kernels()
 {
-    cudaError_t e = configure_one<FSmall>();
-    if (e != cudaSuccess) return e;
-    return configure_one<FWide>();
+    cudaError_t e = configure_one<FSplit>();
+    if (e == cudaSuccess) e = configure_one<FSmall>();
+    if (e == cudaSuccess) e = configure_one<FWide>();
+    return e;
 }
 
 bool fused_step_uses_wide_tiles(int64_t h, int64_t count, int sms)
@@ -348,7 +394,9 @@ cudaError_t launch_fused_step(const Node *tab, const Launch &op, const Bases &ba
     const bool wide = fused_step_uses_wide_tiles(op.h, op.count, sm_count);
     for (int64_t item0 = 0; item0 < op.count; item0 += kMaxItemsPerLaunch) {
         const int64_t zn = op.count - item0 < kMaxItemsPerLaunch ? op.count - item0 : kMaxItemsPerLaunch;
+        const int64_t small_tiles = ((op.h + FSmall::TM - 1) / FSmall::TM) * ((op.h + FSmall::TN - 1) / FSmall::TN) * zn;
         if (wide) launch_one<FWide>(parents, bases, int(op.h), item0, zn, op.peel_fused, stream);
+        else if (small_tiles <= sm_count) launch_one<FSplit>(parents, bases, int(op.h), item0, zn, op.peel_fused, stream);
         else launch_one<FSmall>(parents, bases, int(op.h), item0, zn, op.peel_fused, stream);
         ++*launched;
     }

@@ -264,12 +264,12 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         level += g;
     }
     if (fused) {
-        // one kernel for the whole deepest step: tiles of 16 x 32 positions, h / 16 slabs each; 0.84 us per slab for a
-        // CTA alone on its SM, 1.25 us when two share one (measured at h = 256, 384, 512)
+        // one kernel for the whole deepest step: tiles of 16 x 32 positions, h / 16 slabs each; 0.72 us per slab for a
+        // CTA alone on its SM (two warps per tile), 1.25 us when two share one (measured at h = 256, 384, 512)
         const double h = double(sizes[L]);
         const double tiles = double((sizes[L] + 15) / 16) * double((sizes[L] + 31) / 32) * visits / sequential;
         const double slabs = double((sizes[L] + 15) / 16);
-        const double per_launch = tiles <= kNominalSMs ? slabs * 0.84 : double(int64_t((tiles + 2 * kNominalSMs - 1) / (2 * kNominalSMs))) * slabs * 1.25;
+        const double per_launch = tiles <= kNominalSMs ? slabs * 0.72 : double(int64_t((tiles + 2 * kNominalSMs - 1) / (2 * kNominalSMs))) * slabs * 1.25;
         out.product_us += per_launch * sequential;
         out.product_flops += visits * 7.0 * 2.0 * h * h * h;
         out.launches += sequential;

@@ -248,15 +248,14 @@ FUSED, UNFUSED = binding.STRASSEN_FLAG_FUSED_STEP, binding.STRASSEN_FLAG_NO_FUSE
     (1000, 125, "DBB", 1, "int8"), (520, 65, "BDB", 2, "int8"), (771, 96, "BBB", 1, "int8"),
     (4096, 512, "BBB", 1, "uniform"),
 ])
-def test_fused_step_gives_the_bits_of_the_three_launch_path(n, cutoff, sched, batch, dist):
+def test_fused_step_agrees_with_the_three_launch_path(n, cutoff, sched, batch, dist):
     A, B = inputs.pair(n, dist, 40 + n, device="cuda", batch=None if batch == 1 else batch)
     fused = run_plan(n, cutoff, sched, A, B, batch=batch, flags=FUSED)
     plain = run_plan(n, cutoff, sched, A, B, batch=batch, flags=UNFUSED)
-    base = oracle.level_sizes(n, cutoff)[-1]
-    if dist == "int8" or not 1 <= base % 64 <= 8:
-        assert torch.equal(fused, plain)             # same operations in the same order on every element
-    else:       # the three-launch path sums the last 1..8 rows / columns of such a base product in another order
-        assert float((fused - plain).abs().max()) <= 1e-3 * bound(n, A, B)
+    if dist == "int8":
+        assert torch.equal(fused, plain)             # same operations on every element, exact on integers
+    else:       # the inner dimension is summed in another order (two partial sums per product; thin remainders)
+        assert float((fused - plain).abs().max()) <= 1e-4 * bound(n, A, B)
     p = Plan(n, cutoff, sched, batch=batch, flags=FUSED)
     assert p.launches_by_kind()["fused_step"] >= 1 and p.launches_by_kind()["gemm"] == 0
     p.close()
