@@ -97,6 +97,12 @@ typedef struct strassen_options {
 #define STRASSEN_FLAG_FUSED_STEP 64
 #define STRASSEN_FLAG_NO_FUSED_STEP 128
 
+/* A DFS step folds each sub-problem's product Q_j into the quadrants of C [Algorithm 1, "locally compute
+ * contribution of Q_i to C"].  Where the sub-problem ends in a one-level recombination pass (a BFS step below
+ * it, even size), that pass does the fold itself and Q_j never reaches memory; NO_DFS_FOLD keeps the separate pass
+ * (write Q_j, read it back, update C) everywhere.  Same operations on every element either way. */
+#define STRASSEN_FLAG_NO_DFS_FOLD 256
+
 /* Replay the plan's launch list as one CUDA graph: the first strassen_dgemm call with a given
  * (A, B, C, workspace) captures the launches on an internal stream and instantiates the graph; that
  * call and every later one with the same pointers costs a single graph launch on the caller's

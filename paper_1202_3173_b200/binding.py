@@ -21,6 +21,7 @@ STRASSEN_FLAG_SCALE_INSIDE = 16
 STRASSEN_FLAG_TWO_LEVEL_PASSES = 32
 STRASSEN_FLAG_FUSED_STEP = 64
 STRASSEN_FLAG_NO_FUSED_STEP = 128
+STRASSEN_FLAG_NO_DFS_FOLD = 256
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SCHEDULE", -3: "WORKSPACE_TOO_SMALL", -4: "ALIAS",
                 -5: "MISALIGNED", -6: "CUDA_ERROR", -7: "OUT_OF_MEMORY"}
 K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_SCALE, K_FUSED_STEP, K_COUNT = range(9)

@@ -11,6 +11,7 @@
 // products in registers: 343 q^2 words in, 64 q^2 out.  Both use the same operations in the same
 // order as the single-level kernels, so results are bit-identical.
 #include "kernels.h"
+#include "fold.cuh"
 
 namespace strassen {
 
@@ -161,9 +162,13 @@ template <int N, class Product, class Emit> __device__ __forceinline__ void u_ch
     emit(1, out);
 }
 
+template <bool FOLD>
 __global__ void __launch_bounds__(TX3 *TY3) recombine3_kernel(const Node *__restrict__ parents, Bases bases, Regions3 reg3,
-                                                              int q, int item0, int peel)
+                                                              int q, int item0, int peel, const Node *__restrict__ dfs_parents,
+                                                              int fold, int fold_peel)
 {
+    // FOLD (fold != 0): the parents are the sub-problems j = fold - 1 of a DFS step one level up; their products are folded
+    // into the C quadrants of those DFS parents instead of being written
     // last parent first: its products are the ones the preceding kernel wrote last, so they are still in L2
     const int par = item0 + (gridDim.z - 1 - blockIdx.z);
     const int c = blockIdx.x * TX3 + threadIdx.x, r = blockIdx.y * TY3 + threadIdx.y;
@@ -173,6 +178,8 @@ __global__ void __launch_bounds__(TX3 *TY3) recombine3_kernel(const Node *__rest
     const int64_t ldc = cc.ld;
     const double *great = bases.p[BASE_WS] + reg3.great_q + int64_t(par) * 343 * reg3.great_mat + int64_t(r) * reg3.great_ld + c;
     const int64_t mat = reg3.great_mat;
+    FoldTarget ft{};
+    if (FOLD) ft = fold_target(dfs_parents[par], bases, 8 * q, fold - 1, fold_peel);
     // peel != 0: parent of odd size 8q + 1; every entry also gets A[row][8q] * B[8q][col], the rank-one
     // term of the peeled split
     const double *acol = nullptr, *brow = nullptr;
@@ -214,7 +221,8 @@ __global__ void __launch_bounds__(TX3 *TY3) recombine3_kernel(const Node *__rest
                     const int bb = (quad & 1) * 4 + v;
                     double val = b[u][v];
                     if (peel) val = fma(av, brow[bb * q], val);
-                    C[(int64_t(a) * q + r) * ldc + bb * q + c] = val;
+                    if (FOLD) fold_emit<1>(ft, a * q + r, bb * q + c, val);
+                    else C[(int64_t(a) * q + r) * ldc + bb * q + c] = val;
                 }
             }
         });
@@ -244,7 +252,12 @@ cudaError_t launch_recombine3(const Node *tab, const Launch &op, const Bases &ba
     const int64_t total = op.count, q = op.h / 4;
     FOR_CHUNKS3(total) {
         const dim3 grid(unsigned((q + TX3 - 1) / TX3), unsigned((q + TY3 - 1) / TY3), unsigned(zn));
-        recombine3_kernel<<<grid, block, 0, stream>>>(tab + op.parent_tab, bases, op.reg3, int(q), int(item0), op.peel_fused);
+        if (op.fold)
+            recombine3_kernel<true><<<grid, block, 0, stream>>>(tab + op.parent_tab, bases, op.reg3, int(q), int(item0), op.peel_fused,
+                                                                tab + op.fold_tab, op.fold, op.fold_peel);
+        else
+            recombine3_kernel<false><<<grid, block, 0, stream>>>(tab + op.parent_tab, bases, op.reg3, int(q), int(item0), op.peel_fused,
+                                                                 nullptr, 0, 0);
         ++*launched;
     }
     return cudaGetLastError();

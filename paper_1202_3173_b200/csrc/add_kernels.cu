@@ -8,6 +8,7 @@
 // each thread handles 4 rows (stride 4) and VEC adjacent columns, issuing all of its loads
 // before the arithmetic so that 4 x (number of input streams) requests are in flight.
 #include "kernels.h"
+#include "fold.cuh"
 
 namespace strassen {
 
@@ -15,30 +16,6 @@ namespace {
 
 constexpr int TX = 64, TY = 4, ROWS_PER_THREAD = 4, TILE_ROWS = TY * ROWS_PER_THREAD;
 constexpr int MAX_Z = kMaxItemsPerLaunch;   // items per launch (gridDim.z limit is 65535)
-
-template <int VEC> struct Vec;
-template <> struct Vec<1> {
-    using type = double;
-    static __device__ __forceinline__ double ld(const double *p) { return __ldcs(p); }
-    static __device__ __forceinline__ double ldk(const double *p) { return *p; }
-    static __device__ __forceinline__ void st(double *p, double v) { *p = v; }
-    static __device__ __forceinline__ double add(double a, double b) { return a + b; }
-    static __device__ __forceinline__ double sub(double a, double b) { return a - b; }
-    static __device__ __forceinline__ double neg(double a) { return -a; }
-    static __device__ __forceinline__ double fma1(double a, double b, double v) { return fma(a, b, v); }
-};
-template <> struct Vec<2> {
-    using type = double2;
-    static __device__ __forceinline__ double2 ld(const double *p) { return __ldcs(reinterpret_cast<const double2 *>(p)); }
-    static __device__ __forceinline__ double2 ldk(const double *p) { return *reinterpret_cast<const double2 *>(p); }
-    static __device__ __forceinline__ void st(double *p, double2 v) { *reinterpret_cast<double2 *>(p) = v; }
-    static __device__ __forceinline__ double2 add(double2 a, double2 b) { return make_double2(a.x + b.x, a.y + b.y); }
-    static __device__ __forceinline__ double2 sub(double2 a, double2 b) { return make_double2(a.x - b.x, a.y - b.y); }
-    static __device__ __forceinline__ double2 neg(double2 a) { return make_double2(-a.x, -a.y); }
-    static __device__ __forceinline__ double2 fma1(double a, double2 b, double2 v) { return make_double2(fma(a, b.x, v.x), fma(a, b.y, v.y)); }
-};
-
-__device__ __forceinline__ double *resolve(const Bases &bases, const Operand &x) { return base_ptr(bases, x.base) + x.off; }
 
 // ---------------------------------------------------------------------------------------
 // BFS operand formation.  item = 2 * parent + side; side 0 forms T2..T5 from the quadrants
@@ -110,11 +87,14 @@ __global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict
 //   U1 = Q0 + Q3   U2 = U1 + Q4   U3 = U1 + Q2
 //   C11 = Q0 + Q1  C12 = U3 + Q5  C21 = U2 - Q6  C22 = U2 + Q2
 // ---------------------------------------------------------------------------------------
-template <int VEC, int RPT>
+template <int VEC, int RPT, bool FOLD>
 __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__restrict__ parents,
                                                                const Node *__restrict__ children, Bases bases,
-                                                               int h, int item0, int peel)
+                                                               int h, int item0, int peel, const Node *__restrict__ dfs_parents,
+                                                               int fold, int fold_peel)
 {
+    // FOLD (fold != 0): the parents are the sub-problems j = fold - 1 of a DFS step one level up; their products are not
+    // written but folded into the C quadrants of those DFS parents (size 2 * (2h)).
     // peel != 0: the parent has odd size 2h + 1; the rank-one term A[r][2h] * B[2h][c] of the peeled split
     // is added to every entry on its way out (saves a read-modify-write pass over C).
     using V = Vec<VEC>;
@@ -142,6 +122,8 @@ __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__res
     const Operand cc = parents[par].c;
     double *C = resolve(bases, cc);
     const int64_t ldc = cc.ld, hq = int64_t(h) * ldc;
+    FoldTarget ft{};
+    if (FOLD) ft = fold_target(dfs_parents[par], bases, 2 * h, fold - 1, fold_peel);
     const int r0 = blockIdx.y * (TY * RPT) + threadIdx.y;
     constexpr int RP = RPT < 2 ? RPT : 2;   // rows per pass: 14 vectors in flight per thread
 #pragma unroll
@@ -170,10 +152,17 @@ __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__res
                     c11 = V::fma1(a0, b0, c11); c12 = V::fma1(a0, b1, c12);
                     c21 = V::fma1(a1, b0, c21); c22 = V::fma1(a1, b1, c22);
                 }
-                V::st(o, c11);
-                V::st(o + h, c12);
-                V::st(o + hq, c21);
-                V::st(o + hq + h, c22);
+                if (FOLD) {
+                    fold_emit<VEC>(ft, r, c, c11);
+                    fold_emit<VEC>(ft, r, c + h, c12);
+                    fold_emit<VEC>(ft, r + h, c, c21);
+                    fold_emit<VEC>(ft, r + h, c + h, c22);
+                } else {
+                    V::st(o, c11);
+                    V::st(o + h, c12);
+                    V::st(o + hq, c21);
+                    V::st(o + hq + h, c22);
+                }
             }
         }
     }
@@ -186,8 +175,10 @@ __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__res
 template <int VEC>
 __global__ void __launch_bounds__(TX *TY) form_one_kernel(const Node *__restrict__ parents,
                                                           const Node *__restrict__ children, Bases bases, int h,
-                                                          int j, int sides, int item0)
+                                                          int j, int sides, int item0, int chain)
 {
+    // chain != 0: the slot still holds the sum formed for the sub-problem before this one, and the new sum grows out
+    // of it in place: T3 = T2 - A11, T5 = A12 - T3, S3 = B22 - S2, S6 = S3 - B21 (Appendix A's own chain).
     using V = Vec<VEC>;
     using T = typename V::type;
     const int item = item0 + blockIdx.z;
@@ -202,14 +193,19 @@ __global__ void __launch_bounds__(TX *TY) form_one_kernel(const Node *__restrict
     double *O = resolve(bases, y);
     const int64_t ld = x.ld, hq = int64_t(h) * ld, ldo = y.ld;
     const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
-    const int which = side * 8 + j;
+    const int which = side * 8 + j + (chain ? 16 : 0);
 #pragma unroll
     for (int i = 0; i < ROWS_PER_THREAD; ++i) {
         const int r = r0 + i * TY;
         if (r >= h) continue;
         const double *q = X + int64_t(r) * ld + c;
+        double *slot = O + int64_t(r) * ldo + c;
         T v;
         switch (which) {
+        case 16 + 3: v = V::sub(V::ldk(slot), V::ld(q)); break;                 // T3 = T2 - A11
+        case 16 + 5: v = V::sub(V::ld(q + h), V::ldk(slot)); break;             // T5 = A12 - T3
+        case 16 + 11: v = V::sub(V::ld(q + hq + h), V::ldk(slot)); break;       // S3 = B22 - S2
+        case 16 + 14: v = V::sub(V::ldk(slot), V::ld(q + hq)); break;           // S6 = S3 - B21
         case 2: v = V::add(V::ld(q + hq), V::ld(q + hq + h)); break;                                   // T2
         case 3: v = V::sub(V::add(V::ld(q + hq), V::ld(q + hq + h)), V::ld(q)); break;                 // T3
         case 4: v = V::sub(V::ld(q), V::ld(q + hq)); break;                                            // T4
@@ -219,14 +215,13 @@ __global__ void __launch_bounds__(TX *TY) form_one_kernel(const Node *__restrict
         case 12: v = V::sub(V::ld(q + hq + h), V::ld(q + h)); break;                                   // S4
         default: v = V::sub(V::sub(V::ld(q + hq + h), V::sub(V::ld(q + h), V::ld(q))), V::ld(q + hq)); break;  // S6
         }
-        V::st(O + int64_t(r) * ldo + c, v);
+        V::st(slot, v);
     }
 }
 
 // ---------------------------------------------------------------------------------------
-// DFS fold of Q_j into C (Algorithm 1: "locally compute contribution of Q_i to C"), the flat
-// form of the U chain:  C11 = Q0+Q1, C12 = Q0+Q3+Q2+Q5, C21 = Q0+Q3+Q4-Q6, C22 = Q0+Q3+Q4+Q2.
-// Q0 writes all four quadrants (first touch), later Q_j read-modify-write theirs.
+// DFS fold of Q_j into C as a pass of its own, for sub-problems that do not end in a recombination
+// pass (a leaf product, a DFS step or a fused step below): reads the Q_j the sub-problem wrote.
 // ---------------------------------------------------------------------------------------
 template <int VEC>
 __global__ void __launch_bounds__(TX *TY) accumulate_kernel(const Node *__restrict__ parents,
@@ -234,44 +229,19 @@ __global__ void __launch_bounds__(TX *TY) accumulate_kernel(const Node *__restri
                                                             int j, int item0, int peel)
 {
     using V = Vec<VEC>;
-    using T = typename V::type;
     const int par = item0 + blockIdx.z;
     const int c = (blockIdx.x * TX + threadIdx.x) * VEC;
     if (c >= h) return;
-    const Operand qq = children[par].c, cc = parents[par].c;
+    const Operand qq = children[par].c;
     const double *Q = resolve(bases, qq);
-    double *C = resolve(bases, cc);
-    const int64_t ldq = qq.ld, ldc = cc.ld, hq = int64_t(h) * ldc;
+    const int64_t ldq = qq.ld;
+    const FoldTarget ft = fold_target(parents[par], bases, h, j, peel);
     const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
 #pragma unroll
     for (int i = 0; i < ROWS_PER_THREAD; ++i) {
         const int r = r0 + i * TY;
         if (r >= h) continue;
-        const T q = V::ld(Q + int64_t(r) * ldq + c);
-        double *o = C + int64_t(r) * ldc + c;
-        double *c11 = o, *c12 = o + h, *c21 = o + hq, *c22 = o + hq + h;
-        switch (j) {
-        case 0:
-            if (peel) {     // odd parent: the first touch also carries the rank-one term of the peeled split
-                const Operand pa = parents[par].a, pb = parents[par].b;
-                const double *acol = resolve(bases, pa) + 2 * h;
-                const double *brow = resolve(bases, pb) + int64_t(2 * h) * pb.ld + c;
-                const double a0 = acol[int64_t(r) * pa.ld], a1 = acol[int64_t(r + h) * pa.ld];
-                const T b0 = V::ldk(brow), b1 = V::ldk(brow + h);
-                V::st(c11, V::fma1(a0, b0, q)); V::st(c12, V::fma1(a0, b1, q));
-                V::st(c21, V::fma1(a1, b0, q)); V::st(c22, V::fma1(a1, b1, q));
-            } else {
-                V::st(c11, q); V::st(c12, q); V::st(c21, q); V::st(c22, q);
-            }
-            break;
-        case 1: V::st(c11, V::add(V::ldk(c11), q)); break;
-        case 2: V::st(c12, V::add(V::ldk(c12), q)); V::st(c22, V::add(V::ldk(c22), q)); break;
-        case 3: V::st(c12, V::add(V::ldk(c12), q)); V::st(c21, V::add(V::ldk(c21), q));
-                V::st(c22, V::add(V::ldk(c22), q)); break;
-        case 4: V::st(c21, V::add(V::ldk(c21), q)); V::st(c22, V::add(V::ldk(c22), q)); break;
-        case 5: V::st(c12, V::add(V::ldk(c12), q)); break;
-        default: V::st(c21, V::sub(V::ldk(c21), q)); break;
-        }
+        fold_emit<VEC>(ft, r, c, V::ld(Q + int64_t(r) * ldq + c));
     }
 }
 
@@ -374,9 +344,10 @@ __global__ void __launch_bounds__(TX *TY) form2_kernel(const Node *__restrict__ 
 // registers, never written), and those give the parent's C at its 16 block positions:
 // 12.25 h^2 read + 4 h^2 written instead of 19.25 h^2 + 11 h^2.
 // ---------------------------------------------------------------------------------------
-template <int VEC>
+template <int VEC, bool FOLD>
 __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restrict__ parents, Bases bases, Regions2 reg,
-                                                            int q, int item0, int peel)
+                                                            int q, int item0, int peel, const Node *__restrict__ dfs_parents,
+                                                            int fold, int fold_peel)
 {
     using V = Vec<VEC>;
     using T = typename V::type;
@@ -389,6 +360,8 @@ __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restri
     const int64_t ldc = cc.ld, gld = reg.grand_ld;
     const double *grand = bases.p[BASE_WS] + reg.grand_q + int64_t(par) * 49 * reg.grand_mat;
     const int r0 = blockIdx.y * TILE_ROWS + threadIdx.y;
+    FoldTarget ft{};
+    if (FOLD) ft = fold_target(dfs_parents[par], bases, 4 * q, fold - 1, fold_peel);     // see recombine_bfs_kernel
     // peel != 0: parent of odd size 4q + 1; add A[row][4q] * B[4q][col] to every entry (see recombine_bfs_kernel)
     const double *acol = nullptr;
     int64_t lda = 0;
@@ -437,10 +410,18 @@ __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restri
                     c11 = V::fma1(a0, bv[v], c11); c12 = V::fma1(a0, bv[2 + v], c12);
                     c21 = V::fma1(a1, bv[v], c21); c22 = V::fma1(a1, bv[2 + v], c22);
                 }
-                V::st(o, c11);
-                V::st(o + h, c12);
-                V::st(o + h * ldc, c21);
-                V::st(o + h * ldc + h, c22);
+                if (FOLD) {
+                    const int R = u * q + r, Cc = v * q + c;
+                    fold_emit<VEC>(ft, R, Cc, c11);
+                    fold_emit<VEC>(ft, R, Cc + int(h), c12);
+                    fold_emit<VEC>(ft, R + int(h), Cc, c21);
+                    fold_emit<VEC>(ft, R + int(h), Cc + int(h), c22);
+                } else {
+                    V::st(o, c11);
+                    V::st(o + h, c12);
+                    V::st(o + h * ldc, c21);
+                    V::st(o + h * ldc + h, c22);
+                }
             }
     }
 }
@@ -474,154 +455,106 @@ __global__ void __launch_bounds__(256) peel_rank1_kernel(const Node *__restrict_
 // Thin products: a few columns or a few rows of C = A.B of one node, over the full inner
 // dimension K.  They serve the peeled last column / row (one of each) and the ragged remainder of
 // base products whose size is a few elements past a multiple of the GEMM tile (e.g. 771 = 768 + 3).
-// Both read one operand in full once; summation order is fixed (bit-reproducible).
-
-// Columns [c0, c0 + nc) of C for rows [0, rows): each warp owns 4 rows, lanes stride over k; the nc
-// columns of B are staged through shared memory in chunks of TC_CHUNK rows.
-constexpr int TC_ROWS = 32, TC_CHUNK = 512;
-template <int NC>
-__global__ void __launch_bounds__(256) thin_cols_kernel(const Node *__restrict__ nodes, Bases bases, int K, int rows,
-                                                        int c0, int nc, int item0)
+// Both read one operand in full exactly once and are bound by that stream from HBM.  They run on the FP64
+// tensor cores with the operand fragments loaded straight from global memory in the layout mma.sync
+// m8n8k4 wants (no shared-memory staging): a lane's 8-byte load of the large operand shares its 32-byte
+// sector with the three lanes next to it, so every sector fetched is used in full, and 8 to 16 such loads
+// per lane are in flight before the first DMMA.  Summation runs over k ascending: bit-reproducible.
+__device__ __forceinline__ void dmma_thin(double &d0, double &d1, double a, double b)
 {
-    __shared__ double bs[NC][TC_CHUNK];
+    asm("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
+        : "+d"(d0), "+d"(d1)
+        : "d"(a), "d"(b));
+}
+
+constexpr int THIN_WARPS = 4, THIN_STEPS = 8;      // warps per CTA; 4-deep steps per loop iteration
+
+// Columns [c0, c0 + nc) of C for rows [0, rows), nc <= 8: a warp owns 8 rows.  g = lane / 4, q = lane % 4:
+// the lane feeds A[row g][k + q] and B[k + q][column g] and receives C[row g][columns 2q, 2q + 1].
+__global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_kernel(const Node *__restrict__ nodes, Bases bases, int K, int rows,
+                                                                    int c0, int nc, int item0)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
+    const int m0 = (blockIdx.x * THIN_WARPS + warp) * 8;
+    if (m0 >= rows) return;
     const Node nd = nodes[item0 + blockIdx.y];
     const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
-    double *C = resolve(bases, nd.c);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rbase = blockIdx.x * TC_ROWS + warp * 4;
-    double acc[4][NC];
+    const bool row_ok = m0 + g < rows, col_ok = g < nc;
+    const double *a = A + int64_t(row_ok ? m0 + g : 0) * nd.a.ld + q;
+    const double *b = B + int64_t(q) * nd.b.ld + c0 + (col_ok ? g : 0);
+    const int64_t ldb = nd.b.ld;
+    double d0 = 0.0, d1 = 0.0;
+    for (int k0 = 0; k0 < K; k0 += 4 * THIN_STEPS) {
+        double av[THIN_STEPS], bv[THIN_STEPS];
+        if (k0 + 4 * THIN_STEPS <= K) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+            for (int s = 0; s < THIN_STEPS; ++s) av[s] = row_ok ? __ldcs(a + k0 + 4 * s) : 0.0;
 #pragma unroll
-        for (int t = 0; t < NC; ++t) acc[i][t] = 0.0;
-    for (int k0 = 0; k0 < K; k0 += TC_CHUNK) {
-        const int kn = min(TC_CHUNK, K - k0);
-        __syncthreads();
-        for (int e = threadIdx.x; e < kn * NC; e += 256) {
-            const int k = e / NC, t = e % NC;
-            bs[t][k] = t < nc ? B[int64_t(k0 + k) * nd.b.ld + c0 + t] : 0.0;
-        }
-        __syncthreads();
-        // k outer, the warp's 4 rows inner: the staged B values are read from shared memory once per k
-        const double *a0 = A + int64_t(min(rbase, rows - 1)) * nd.a.ld + k0;
-        const int64_t lda = nd.a.ld;
-        const int nrow = min(4, rows - rbase);
-        int k = lane;
-        for (; k + 32 < kn; k += 64) {              // two k per lane and pass: eight loads of A in flight
-            double av[2][4];
+            for (int s = 0; s < THIN_STEPS; ++s) bv[s] = col_ok ? b[int64_t(k0 + 4 * s) * ldb] : 0.0;
+        } else {
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) av[u][i] = i < nrow ? a0[int64_t(i) * lda + k + 32 * u] : 0.0;
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                double bv[NC];
-#pragma unroll
-                for (int t = 0; t < NC; ++t) bv[t] = bs[t][k + 32 * u];
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int t = 0; t < NC; ++t) acc[i][t] = fma(av[u][i], bv[t], acc[i][t]);
+            for (int s = 0; s < THIN_STEPS; ++s) {
+                const bool k_ok = k0 + 4 * s + q < K;
+                av[s] = row_ok && k_ok ? __ldcs(a + k0 + 4 * s) : 0.0;
+                bv[s] = col_ok && k_ok ? b[int64_t(k0 + 4 * s) * ldb] : 0.0;
             }
         }
-        for (; k < kn; k += 32) {
-            double bv[NC];
 #pragma unroll
-            for (int t = 0; t < NC; ++t) bv[t] = bs[t][k];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (i < nrow) {
-                    const double av = a0[int64_t(i) * lda + k];
-#pragma unroll
-                    for (int t = 0; t < NC; ++t) acc[i][t] = fma(av, bv[t], acc[i][t]);
-                }
-            }
-        }
+        for (int s = 0; s < THIN_STEPS; ++s) dmma_thin(d0, d1, av[s], bv[s]);
     }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int r = rbase + i;
-#pragma unroll
-        for (int t = 0; t < NC; ++t) {
-            double v = acc[i][t];
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-            if (lane == 0 && r < rows && t < nc) C[int64_t(r) * nd.c.ld + c0 + t] = v;
-        }
+    if (row_ok) {
+        double *o = resolve(bases, nd.c) + int64_t(m0 + g) * nd.c.ld + c0 + 2 * q;
+        if (2 * q < nc) o[0] = d0;
+        if (2 * q + 1 < nc) o[1] = d1;
     }
 }
 
-// Rows [r0, r0 + nr) of C for columns [0, cols): a thread owns two adjacent columns and one of
-// TR_SLICES interleaved pairs of k; the nr rows of A are staged through shared memory in chunks (read
-// back as broadcast 16-byte pairs), and the slices are summed through shared memory in a fixed order.
-constexpr int TR_COLS = 64, TR_SLICES = 8, TR_CHUNK = 512;
-template <int NR>
-__global__ void __launch_bounds__((TR_COLS / 2) * TR_SLICES) thin_rows_kernel(const Node *__restrict__ nodes, Bases bases,
-                                                                              int K, int cols, int r0, int nr, int item0)
+// Rows [r0, r0 + nr) of C for columns [0, cols), nr <= 8: a warp owns NT adjacent groups of 8 columns.  The lane
+// feeds A[r0 + g][k + q] (zero for g >= nr) and B[k + q][column g of each group].
+template <int NT>
+__global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_kernel(const Node *__restrict__ nodes, Bases bases, int K, int cols,
+                                                                    int r0, int nr, int item0)
 {
-    // one buffer, used first for the staged rows of A and, after the k loop, for the slice sums
-    constexpr int AS_WORDS = NR * TR_CHUNK, PART_WORDS = TR_SLICES * NR * (TR_COLS + 2);
-    __shared__ __align__(16) double buf[AS_WORDS > PART_WORDS ? AS_WORDS : PART_WORDS];
-    double(*as)[TR_CHUNK] = reinterpret_cast<double(*)[TR_CHUNK]>(buf);
-    double(*part)[NR][TR_COLS + 2] = reinterpret_cast<double(*)[NR][TR_COLS + 2]>(buf);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
+    const int n0 = (blockIdx.x * THIN_WARPS + warp) * 8 * NT;
+    if (n0 >= cols) return;
     const Node nd = nodes[item0 + blockIdx.y];
     const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
-    double *C = resolve(bases, nd.c);
-    const int tid = threadIdx.y * (TR_COLS / 2) + threadIdx.x;
-    const int c = blockIdx.x * TR_COLS + 2 * threadIdx.x;
-    const bool c0ok = c < cols, c1ok = c + 1 < cols;
-    const int64_t ldb = nd.b.ld, lda = nd.a.ld;
-    const double *b = B + (c0ok ? c : 0);
-    const int c1 = c1ok ? 1 : 0;
-    double acc[NR][2];
+    const bool row_ok = g < nr;
+    const double *a = A + int64_t(r0 + (row_ok ? g : 0)) * nd.a.ld + q;
+    const int64_t ldb = nd.b.ld;
+    bool col_ok[NT];
+    const double *b[NT];
 #pragma unroll
-    for (int t = 0; t < NR; ++t) acc[t][0] = acc[t][1] = 0.0;
-    for (int k0 = 0; k0 < K; k0 += TR_CHUNK) {
-        const int kn = min(TR_CHUNK, K - k0);
-        __syncthreads();
-        for (int e = tid; e < NR * TR_CHUNK; e += (TR_COLS / 2) * TR_SLICES) {
-            const int t = e / TR_CHUNK, k = e % TR_CHUNK;
-            as[t][k] = (t < nr && k < kn) ? A[int64_t(r0 + t) * lda + k0 + k] : 0.0;
-        }
-        __syncthreads();
-        if (c0ok) {
-            // slice s owns k = 2 s, 2 s + 1, then + 2 TR_SLICES, ...; entries past kn are zero in `as`
-            for (int k = 2 * threadIdx.y; k < kn; k += 2 * TR_SLICES) {
-                const double *bk = b + int64_t(k0 + k) * ldb;
-                const bool k1ok = k + 1 < kn;
-                const double b00 = bk[0], b01 = bk[c1];
-                const double b10 = k1ok ? bk[ldb] : 0.0, b11 = k1ok ? bk[ldb + c1] : 0.0;
-#pragma unroll
-                for (int t = 0; t < NR; ++t) {
-                    const double2 a2 = *reinterpret_cast<const double2 *>(&as[t][k]);
-                    acc[t][0] = fma(a2.x, b00, acc[t][0]);
-                    acc[t][1] = fma(a2.x, b01, acc[t][1]);
-                    acc[t][0] = fma(a2.y, b10, acc[t][0]);
-                    acc[t][1] = fma(a2.y, b11, acc[t][1]);
-                }
-            }
-        }
+    for (int j = 0; j < NT; ++j) {
+        col_ok[j] = n0 + 8 * j + g < cols;
+        b[j] = B + int64_t(q) * ldb + (col_ok[j] ? n0 + 8 * j + g : 0);
     }
-    __syncthreads();    // everyone is done reading the staged rows
+    double d[NT][2];
 #pragma unroll
-    for (int t = 0; t < NR; ++t) {
-        part[threadIdx.y][t][2 * threadIdx.x] = acc[t][0];
-        part[threadIdx.y][t][2 * threadIdx.x + 1] = acc[t][1];
+    for (int j = 0; j < NT; ++j) d[j][0] = d[j][1] = 0.0;
+    for (int k0 = 0; k0 < K; k0 += 4 * THIN_STEPS) {
+        double av[THIN_STEPS], bv[THIN_STEPS][NT];
+        const bool full = k0 + 4 * THIN_STEPS <= K;
+#pragma unroll
+        for (int s = 0; s < THIN_STEPS; ++s) {
+            const bool k_ok = full || k0 + 4 * s + q < K;
+#pragma unroll
+            for (int j = 0; j < NT; ++j) bv[s][j] = col_ok[j] && k_ok ? __ldcs(b[j] + int64_t(k0 + 4 * s) * ldb) : 0.0;
+            av[s] = row_ok && k_ok ? a[k0 + 4 * s] : 0.0;
+        }
+#pragma unroll
+        for (int s = 0; s < THIN_STEPS; ++s)
+#pragma unroll
+            for (int j = 0; j < NT; ++j) dmma_thin(d[j][0], d[j][1], av[s], bv[s][j]);
     }
-    __syncthreads();
-    if (threadIdx.y == 0 && c0ok) {
+    if (row_ok) {
+        double *o = resolve(bases, nd.c) + int64_t(r0 + g) * nd.c.ld;
 #pragma unroll
-        for (int t = 0; t < NR; ++t) {
-            double v0 = 0.0, v1 = 0.0;
-#pragma unroll
-            for (int i = 0; i < TR_SLICES; ++i) {
-                v0 += part[i][t][2 * threadIdx.x];
-                v1 += part[i][t][2 * threadIdx.x + 1];
-            }
-            if (t < nr) {
-                C[int64_t(r0 + t) * nd.c.ld + c] = v0;
-                if (c1ok) C[int64_t(r0 + t) * nd.c.ld + c + 1] = v1;
-            }
+        for (int j = 0; j < NT; ++j) {
+            const int c = n0 + 8 * j + 2 * q;
+            if (c < cols) o[c] = d[j][0];
+            if (c + 1 < cols) o[c + 1] = d[j][1];
         }
     }
 }
@@ -690,6 +623,18 @@ cudaError_t launch_form(const Node *tab, const Launch &op, const Bases &bases, b
     return cudaGetLastError();
 }
 
+template <int VEC, int RPT>
+void launch_recombine_as(const dim3 &grid, const dim3 &block, cudaStream_t stream, const Node *tab, const Launch &op, const Bases &bases,
+                         int64_t item0)
+{
+    const Node *par = tab + op.parent_tab, *kid = tab + op.child_tab;
+    if (op.fold)
+        recombine_bfs_kernel<VEC, RPT, true><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused,
+                                                                        tab + op.fold_tab, op.fold, op.fold_peel);
+    else
+        recombine_bfs_kernel<VEC, RPT, false><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused, nullptr, 0, 0);
+}
+
 cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
                              int *launched)
 {
@@ -698,14 +643,15 @@ cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bas
     FOR_CHUNKS(total) {
         const int v = vec ? 2 : 1;
         const dim3 grid = tile_grid(op.h, v, zn);
-        const Node *par = tab + op.parent_tab, *kid = tab + op.child_tab;
-        if (small_grid(grid)) {
+        // folding passes also take one row per thread: their read-modify-write of C is a second round trip to memory
+        // behind the loads of the products, and four times the CTAs keep enough of both in flight
+        if (small_grid(grid) || op.fold) {
             const dim3 g1(grid.x, unsigned((op.h + TY - 1) / TY), grid.z);
-            if (vec) recombine_bfs_kernel<2, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
-            else recombine_bfs_kernel<1, 1><<<g1, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
+            if (vec) launch_recombine_as<2, 1>(g1, block, stream, tab, op, bases, item0);
+            else launch_recombine_as<1, 1>(g1, block, stream, tab, op, bases, item0);
         } else {
-            if (vec) recombine_bfs_kernel<2, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
-            else recombine_bfs_kernel<1, ROWS_PER_THREAD><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused);
+            if (vec) launch_recombine_as<2, ROWS_PER_THREAD>(grid, block, stream, tab, op, bases, item0);
+            else launch_recombine_as<1, ROWS_PER_THREAD>(grid, block, stream, tab, op, bases, item0);
         }
         ++*launched;
     }
@@ -726,18 +672,26 @@ cudaError_t launch_form2(const Node *tab, const Launch &op, const Bases &bases, 
     return cudaGetLastError();
 }
 
+template <int VEC>
+void launch_recombine2_as(const dim3 &grid, const dim3 &block, cudaStream_t stream, const Node *tab, const Launch &op, const Bases &bases,
+                          int64_t q, int64_t item0)
+{
+    if (op.fold)
+        recombine2_kernel<VEC, true><<<grid, block, 0, stream>>>(tab + op.parent_tab, bases, op.reg, int(q), int(item0), op.peel_fused,
+                                                                tab + op.fold_tab, op.fold, op.fold_peel);
+    else
+        recombine2_kernel<VEC, false><<<grid, block, 0, stream>>>(tab + op.parent_tab, bases, op.reg, int(q), int(item0), op.peel_fused,
+                                                                 nullptr, 0, 0);
+}
+
 cudaError_t launch_recombine2(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
                               int *launched)
 {
     const dim3 block(TX, TY);
     const int64_t total = op.count, q = op.h / 2;
     FOR_CHUNKS(total) {
-        if (vec)
-            recombine2_kernel<2><<<tile_grid(q, 2, zn), block, 0, stream>>>(tab + op.parent_tab, bases, op.reg, int(q),
-                                                                           int(item0), op.peel_fused);
-        else
-            recombine2_kernel<1><<<tile_grid(q, 1, zn), block, 0, stream>>>(tab + op.parent_tab, bases, op.reg, int(q),
-                                                                           int(item0), op.peel_fused);
+        if (vec) launch_recombine2_as<2>(tile_grid(q, 2, zn), block, stream, tab, op, bases, q, item0);
+        else launch_recombine2_as<1>(tile_grid(q, 1, zn), block, stream, tab, op, bases, q, item0);
         ++*launched;
     }
     return cudaGetLastError();
@@ -754,10 +708,10 @@ cudaError_t launch_form_one(const Node *tab, const Launch &op, const Bases &base
     FOR_CHUNKS(total) {
         if (vec)
             form_one_kernel<2><<<tile_grid(op.h, 2, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
-                                                                            bases, int(op.h), j, sides, int(item0));
+                                                                            bases, int(op.h), j, sides, int(item0), op.chain);
         else
             form_one_kernel<1><<<tile_grid(op.h, 1, zn), block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab,
-                                                                            bases, int(op.h), j, sides, int(item0));
+                                                                            bases, int(op.h), j, sides, int(item0), op.chain);
         ++*launched;
     }
     return cudaGetLastError();
@@ -785,11 +739,8 @@ cudaError_t launch_thin_cols(const Node *nodes, const Bases &bases, int K, int r
 {
     const int64_t total = count;
     FOR_CHUNKS(total) {
-        const dim3 grid((rows + TC_ROWS - 1) / TC_ROWS, unsigned(zn));
-        if (nc <= 1) thin_cols_kernel<1><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
-        else if (nc <= 2) thin_cols_kernel<2><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
-        else if (nc <= 4) thin_cols_kernel<4><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
-        else thin_cols_kernel<8><<<grid, 256, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        const dim3 grid((rows + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
+        thin_cols_kernel<<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
         ++*launched;
     }
     return cudaGetLastError();
@@ -799,12 +750,16 @@ cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int c
                              cudaStream_t stream, int *launched)
 {
     const int64_t total = count;
+    // two groups of 8 columns per warp (128-byte runs of B) where that still leaves every SM a few dozen warps
+    const bool two = (int64_t(cols + 15) / 16) * count >= 32 * int64_t(kNominalSMs);
     FOR_CHUNKS(total) {
-        const dim3 grid((cols + TR_COLS - 1) / TR_COLS, unsigned(zn)), block(TR_COLS / 2, TR_SLICES);
-        if (nr <= 1) thin_rows_kernel<1><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
-        else if (nr <= 2) thin_rows_kernel<2><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
-        else if (nr <= 4) thin_rows_kernel<4><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
-        else thin_rows_kernel<8><<<grid, block, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+        if (two) {
+            const dim3 grid((cols + 16 * THIN_WARPS - 1) / (16 * THIN_WARPS), unsigned(zn));
+            thin_rows_kernel<2><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+        } else {
+            const dim3 grid((cols + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
+            thin_rows_kernel<1><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+        }
         ++*launched;
     }
     return cudaGetLastError();

@@ -290,6 +290,7 @@ strassen_plan *create(const strassen_options &o)
         return nullptr;
     }
     d.fused_step = (o.flags & STRASSEN_FLAG_NO_FUSED_STEP) ? 2 : (o.flags & STRASSEN_FLAG_FUSED_STEP) ? 1 : 0;
+    d.no_dfs_fold = (o.flags & STRASSEN_FLAG_NO_DFS_FOLD) != 0;
     d.max_fused_levels = (o.flags & STRASSEN_FLAG_SINGLE_LEVEL_PASSES) ? 1 : (o.flags & STRASSEN_FLAG_TWO_LEVEL_PASSES) ? 2 : 3;
     p->use_graph = (o.flags & STRASSEN_FLAG_CUDA_GRAPH) != 0;
     p->host_pipeline = (o.flags & STRASSEN_FLAG_HOST_PIPELINE) != 0;

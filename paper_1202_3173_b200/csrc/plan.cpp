@@ -170,7 +170,12 @@ struct Builder {
             }
         } else {
             const int64_t t_base = lv.ws_off, s_base = lv.ws_off + N * mat, q_base = lv.ws_off + 2 * N * mat;
-            for (int j = 0; j < 7; ++j) {
+            // Sub-problems in an order that lets each sum grow out of the one before it in the same slot:
+            // T2 -> T3 = T2 - A11 -> T5 = A12 - T3, S2 -> S3 = B22 - S2 -> S6 = S3 - B21, then T4, S4 from the quadrants
+            // (24 h^2 words instead of 30; same operations as Appendix A's chain).  Q0 stays first: its fold writes C.
+            static constexpr int kOrder[7] = {0, 1, 2, 3, 5, 6, 4};
+            for (int step = 0; step < 7; ++step) {
+                const int j = kOrder[step];
                 std::vector<Node> kids(static_cast<size_t>(N), Node{});
                 for (int64_t q = 0; q < N; ++q) {
                     const Node nd = p->nodes[tab + q];
@@ -184,10 +189,29 @@ struct Builder {
                 Launch f{};
                 f.kind = OP_FORM_ONE; f.level = level; f.j = j; f.vec_ok = parents_even;
                 f.parent_tab = tab; f.child_tab = ctab; f.count = N; f.m = lv.m; f.h = h;
+                f.chain = (j == 3 || j == 5 || j == 6);
+               
                 if (kTQuad[j] < 0 || kSQuad[j] < 0) p->launches.push_back(f);   // j = 0, 1 need no sums
                 build(level + 1, ctab, N);
+                if (!err.empty()) return;
+                // Where the sub-problem ends in a one-level recombination pass (even size), that pass folds the product
+                // into this level's C quadrants itself: Q_j is neither written nor read back.  (The two- and three-level
+                // passes run one CTA per SM and cannot keep such read-modify-writes in flight beside their own loads:
+                // measured slower than a fold pass of its own, so they write Q_j as before.)
+                Launch &last = p->launches.back();
+                const bool folds = !p->no_dfs_fold && (h & 1) == 0 &&
+                                   last.kind == OP_RECOMBINE &&
+                                   last.level == level + 1 && last.parent_tab == ctab;
+                if (folds) {
+                    last.fold = j + 1;
+                    last.fold_peel = lv.peel && j == 0;
+                    last.fold_tab = tab;
+                    last.vec_ok = last.vec_ok && parents_even;
+                    continue;
+                }
                 Launch a = f;
                 a.kind = OP_ACCUMULATE;
+                a.chain = 0;
                 a.peel_fused = lv.peel && j == 0;
                 p->launches.push_back(a);
             }
@@ -246,8 +270,13 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         }
         if (level >= LU) break;                                // the fused deepest step: accounted with the products
         if (sched[level] == 'D') {
-            out.pass_bytes += visits * 57.0 * h * h * 8.0;     // 30 h^2 to form the operands one at a time, 27 h^2 to fold the products
-            out.launches += 12.0 * sequential;
+            // 24 h^2 to form the operands one at a time (each sum grows out of the one before it); the products are folded
+            // into C by the recombination pass below (24 h^2 instead of that pass's h^2 of writes) or, where the
+            // sub-problem does not end in one, written and folded by a pass of their own (31 h^2)
+            const bool folds = level + 1 < LU && upper[level + 1] == 'B' && (sizes[level + 1] & 1) == 0 &&
+                               fused_group_size(sizes, upper, level + 1, 3) == 1;
+            out.pass_bytes += visits * (24.0 + (folds ? 23.0 : 31.0)) * h * h * 8.0;
+            out.launches += (folds ? 5.0 : 12.0) * sequential;
             visits *= 7.0;
             sequential *= 7.0;
             ++level;

@@ -73,6 +73,12 @@ struct Launch {
     int32_t peel_fused;  // recombine / accumulate(j = 0) of an odd-size parent: also add the rank-one term
                          // A[:, m-1] x B[m-1, :] of the peeled split; on OP_PEEL: that term is already in C
     int64_t grand_tab;   // OP_FORM2 / OP_RECOMBINE2: index of the first grandchild node
+    int32_t chain;       // OP_FORM_ONE: the operand is formed from the previous content of its slot (T3 from T2, T5 from T3,
+                         // S3 from S2, S6 from S3) instead of from the quadrants alone
+    int32_t fold;        // OP_RECOMBINE / 2 / 3 whose parents are the sub-problems j of a DFS step one level up: 1 + j, and their
+                         // products are folded straight into the DFS parents' C quadrants instead of being written (0: no fold)
+    int32_t fold_peel;   // ... and the DFS parents have odd size: the first fold (j = 0) carries their rank-one term
+    int64_t fold_tab;    // ... index of the first DFS parent node (DFS parent i owns sub-problem node i)
     Regions2 reg;        // OP_FORM2 / OP_RECOMBINE2 / OP_FORM3 / OP_RECOMBINE3 only
     Regions3 reg3;       // OP_FORM3 / OP_RECOMBINE3 only
 };
@@ -93,6 +99,7 @@ struct PlanDesc {
     int64_t lda = 0, ldb = 0, ldc = 0;
     int64_t stride_a = 0, stride_b = 0, stride_c = 0;
     int max_fused_levels = 3;       // consecutive BFS levels formed / recombined by one pass: up to 3, 2 or 1
+    bool no_dfs_fold = false;       // keep the separate fold pass of a DFS step even where the pass below could fold
     int fused_step = 0;             // deepest BFS step as one kernel: 0 = where the rule says it pays, 1 = always, 2 = never
     bool scale_inside = false, scale_outside = false;   // diagonal scaling (Section 6.1)
     int64_t scale_a_off = 0, scale_b_off = 0, scale_exp_off = 0, scale_ld = 0;   // workspace words / leading dimension

@@ -306,6 +306,24 @@ def test_cuda_graph_replay_matches_launch_by_launch():
         eager.close(); graph.close()
 
 
+@pytest.mark.parametrize("n,cutoff,sched,dist", [
+    (1024, 256, "DB", "uniform"),       # sub-problems end in a one-level recombination
+    (4128, 129, "DBBBB", "uniform"),    # ... one level above a three-level pass
+    (4129, 129, "DBBBB", "int8"),       # odd DFS parent: the first fold carries the rank-one term of the peeled split
+    (1025, 256, "DB", "int8"), (1028, 257, "DB", "normal"),
+    (520, 65, "DDB", "int8"), (1024, 128, "BDB", "uniform"), (260, 65, "DB", "int8"),
+])
+def test_dfs_fold_inside_the_recombination_matches_the_separate_fold_pass(n, cutoff, sched, dist):
+    A, B = inputs.pair(n, dist, 60 + n, device="cuda")
+    through = run_plan(n, cutoff, sched, A, B, flags=UNFUSED)
+    separate = run_plan(n, cutoff, sched, A, B, flags=UNFUSED | binding.STRASSEN_FLAG_NO_DFS_FOLD)
+    assert torch.equal(through, separate)          # the same operations in the same order on every element of C
+    p, q = Plan(n, cutoff, sched, flags=UNFUSED), Plan(n, cutoff, sched, flags=UNFUSED | binding.STRASSEN_FLAG_NO_DFS_FOLD)
+    assert p.launches_by_kind()["accumulate"] < q.launches_by_kind()["accumulate"]
+    p.close(); q.close()
+    check_full(n, cutoff, sched, dist, 60 + n, flags=UNFUSED)
+
+
 def test_schedules_agree_exactly_on_integers():
     A, B = inputs.pair(512, "int8", 41, device="cuda")
     outs = [run_plan(512, 64, s, A, B) for s in ("BBB", "DDD", "BDB", "DBD")]

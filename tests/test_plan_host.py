@@ -182,8 +182,24 @@ def test_launch_lists():
     # DFS on top: 7 x (form_one [not for j = 0, 1], sub-tree, accumulate)
     p = Plan(16384, 512, "DBBBB", flags=single)
     k = p.launches_by_kind()
-    assert k["form_one"] == 5 and k["accumulate"] == 7 and k["gemm"] == 7 and k["form"] == 28 and k["recombine"] == 28
+    # (the recombination pass that ends each sub-problem folds its product into C: no separate fold passes)
+    assert k["form_one"] == 5 and k["accumulate"] == 0 and k["gemm"] == 7 and k["form"] == 28 and k["recombine"] == 28
     assert p.base_products == 7 ** 5
+    p.close()
+    p = Plan(16384, 512, "DBBBB", flags=single | binding.STRASSEN_FLAG_NO_DFS_FOLD)
+    assert p.launches_by_kind()["accumulate"] == 7
+    p.close()
+    # the upper DFS step's sub-problems end in a DFS step (separate fold passes), the lower one's in a recombination
+    p = Plan(1024, 128, "DDB", flags=binding.STRASSEN_FLAG_NO_FUSED_STEP)
+    k = p.launches_by_kind()
+    assert k["accumulate"] == 7 and k["recombine"] == 49
+    p.close()
+    p = Plan(1024, 128, "DDB")          # ... or, by default at this size, in a fused step: separate fold passes again
+    k = p.launches_by_kind()
+    assert k["accumulate"] == 7 + 49 and k["fused_step"] == 49 and k["recombine"] == 0
+    p.close()
+    p = Plan(1026, 256, "DB")           # sub-problems of odd size (513) end in their peeling fix-ups: separate fold passes
+    assert p.launches_by_kind()["accumulate"] == 7
     p.close()
     p = Plan(16384, 512, "DBBBB", flags=two)          # four BFS levels below the DFS step: two pairs
     k = p.launches_by_kind()
