@@ -281,6 +281,36 @@ int strassen_autotune(const strassen_tune_request *request, strassen_tune_entry 
                       int log_capacity, int *log_count);
 
 /*
+ * The two local steps of ONE BFS step spread over seven GPUs [Algorithm 2, BFS(A, B, C, k) with k = 1:
+ * "locally compute T_i, S_i" before the redistribution, "locally compute C from Q_i" after it; Section 3.2 for
+ * the layout that makes both communication-free; Section 3.3 for the message size n^2 / (4 P)].  The exchange
+ * itself (three all-to-alls among the seven ranks: the T blocks, the S blocks, the Q blocks) is the caller's:
+ * the Python layer does it with batched point-to-point operations over NCCL, every block landing in
+ * the receiver's own memory before a kernel reads it.
+ *
+ * Layout.  n even, h = n / 2.  The h rows of every quadrant are cut into seven consecutive blocks of
+ * rows_r = floor(h / 7) + (r < h mod 7) rows; rank r owns block r of all four quadrants of A, B and C.  A share
+ * is a (2 rows_r) x (2 h) row-major matrix with leading dimension ld >= 2 h: [X11_r | X12_r] above [X21_r | X22_r].
+ *
+ * strassen_bfs_form_shares: from the rank's shares of A and B, block r of the seven A-side operands T_0..T_6
+ * and of the seven B-side operands S_0..S_6 [Appendix A], each rows x h with leading dimension ld_out, written
+ * to T_out[j] / S_out[j] (host arrays of seven device pointers): T_out[j] and S_out[j] are what rank r sends to
+ * rank j.  Plain quadrants (T_0 = A11, ...) are copied, since they have to travel too.
+ *
+ * strassen_bfs_combine_shares: from block r of the seven products Q_0..Q_6 (Q_in[j]: rows x h, leading dimension
+ * ldq; what rank j sent to rank r), the rank's share of C through the U-chain [Appendix A].
+ *
+ * Both are asynchronous on `stream`, read every input element once and write every output element once
+ * (HBM-bound), never write their inputs, and allocate nothing.  All pointers are device pointers, 8-byte aligned
+ * (16-byte alignment with even h and leading dimensions selects 16-byte accesses); rows = 0 is allowed and does
+ * nothing.  The sub-product Q_j = T_j . S_j in between is an ordinary strassen_dgemm of size h on rank j.
+ */
+int strassen_bfs_form_shares(int64_t rows, int64_t h, const double *A_share, int64_t lda, const double *B_share,
+                             int64_t ldb, double *const *T_out, double *const *S_out, int64_t ld_out, void *stream);
+int strassen_bfs_combine_shares(int64_t rows, int64_t h, const double *const *Q_in, int64_t ldq, double *C_share,
+                                int64_t ldc, void *stream);
+
+/*
  * strassen_probe_fp64 -- measure the FP64 arithmetic rate of the current device with a
  * register-resident loop (no memory traffic): kind 0 = scalar fused multiply-add, kind 1..4 =
  * the FP64 tensor-core instruction mma.sync m8n8k4 / m16n8k4 / m16n8k8 / m16n8k16.  Runs

@@ -18,6 +18,9 @@ paper that needs no matrix data:
   (a BFS step stores 7 triples S_j,T_j,Q_j of quarter size, a DFS step one),
   ``mem_um_closed_form`` -- Mem_UM = 7 n^2 / P^{2/w0} - 4 n^2 / P at P = 7^k.
 * ``effective_gflops`` -- 2 n^3 / (t 10^9) (Section 5.2).
+* ``bfs_row_blocks``, ``bfs_share``, ``bfs_unshare``, ``bfs_form_shares``,
+  ``bfs_combine_shares`` -- one BFS step spread over seven processors
+  (Algorithm 2 with k = 1; layout of Section 3.2) restated on numpy blocks.
 
 Every function is pinned by tests/test_oracle_*.py to something other than
 itself (closed forms, a hand-worked product, brute-force equality on integer
@@ -259,3 +262,60 @@ def scaled_strassen_winograd(A, B, cutoff, schedule=None, inside: bool = False, 
 def effective_gflops(n: int, seconds: float, batch: int = 1) -> float:
     """Effective GFLOPS = 2 n^3 / (seconds 10^9) (Section 5.2), times the batch size."""
     return 2.0 * n ** 3 * batch / (seconds * 1e9)
+
+
+# ---- one BFS step over P = 7 processors (Algorithm 2, BFS(A, B, C, k) with k = 1) ----------------------
+# Layout (Section 3.2: every processor owns the same part of each quadrant): the h = n / 2 rows of every
+# quadrant are cut into seven consecutive blocks; processor r owns block r of all four quadrants.
+
+def bfs_row_blocks(h: int, P: int = 7):
+    """[(first row, rows)] of the P consecutive row blocks of a quadrant with h rows."""
+    out, start = [], 0
+    for r in range(P):
+        rows = h // P + (1 if r < h % P else 0)
+        out.append((start, rows))
+        start += rows
+    return out
+
+
+def bfs_share(X, r: int, P: int = 7):
+    """Processor r's share of the n x n matrix X: [X11_r | X12_r] stacked on [X21_r | X22_r]."""
+    X = np.asarray(X)
+    h = X.shape[0] // 2
+    start, rows = bfs_row_blocks(h, P)[r]
+    return np.vstack((X[start:start + rows], X[h + start:h + start + rows]))
+
+
+def bfs_unshare(shares, n: int, P: int = 7):
+    """The n x n matrix whose shares are `shares` (inverse of bfs_share over all processors)."""
+    h = n // 2
+    X = np.empty((n, n))
+    for r, (start, rows) in enumerate(bfs_row_blocks(h, P)):
+        X[start:start + rows] = shares[r][:rows]
+        X[h + start:h + start + rows] = shares[r][rows:]
+    return X
+
+
+def bfs_form_shares(A_share, B_share):
+    """Algorithm 2, "locally compute T_i, S_i": block r of the seven operand pairs of Appendix A
+    (typos corrected as in the C oracle) from a processor's shares.  Returns (T, S), lists of 7 blocks."""
+    A_share, B_share = np.asarray(A_share), np.asarray(B_share)
+    rows, h = A_share.shape[0] // 2, A_share.shape[1] // 2
+    a11, a12, a21, a22 = A_share[:rows, :h], A_share[:rows, h:], A_share[rows:, :h], A_share[rows:, h:]
+    b11, b12, b21, b22 = B_share[:rows, :h], B_share[:rows, h:], B_share[rows:, :h], B_share[rows:, h:]
+    t2 = a21 + a22
+    t3 = t2 - a11
+    s2 = b12 - b11
+    s3 = b22 - s2
+    T = [a11.copy(), a12.copy(), t2, t3, a11 - a21, a12 - t3, a22.copy()]
+    S = [b11.copy(), b21.copy(), s2, s3, b22 - b12, b22.copy(), s3 - b21]
+    return T, S
+
+
+def bfs_combine_shares(Q):
+    """Algorithm 2, "locally compute C from Q_i": a processor's share of C from its blocks of Q_0..Q_6."""
+    q = [np.asarray(x) for x in Q]
+    u1 = q[0] + q[3]
+    u2 = u1 + q[4]
+    u3 = u1 + q[2]
+    return np.vstack((np.hstack((q[0] + q[1], u3 + q[5])), np.hstack((u2 - q[6], u2 + q[2]))))

@@ -76,6 +76,8 @@ SYMBOLS = [
     ("strassen_autotune", _int, [ctypes.POINTER(strassen_tune_request), ctypes.POINTER(strassen_tune_entry),
                                  ctypes.POINTER(strassen_tune_entry), _int, ctypes.POINTER(_int)]),
     ("strassen_probe_fp64", _int, [_int, _i64, _vp, _dp]),
+    ("strassen_bfs_form_shares", _int, [_i64, _i64, _vp, _i64, _vp, _i64, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i64, _vp]),
+    ("strassen_bfs_combine_shares", _int, [_i64, _i64, ctypes.POINTER(_vp), _i64, _vp, _i64, _vp]),
     ("strassen_dgemm_static", _int, [_i64, _vp, _vp, _vp, _vp]),
     ("strassen_last_error", _cp, []),
 ]
@@ -225,6 +227,23 @@ def strassen_autotune(n, A, B, C, workspace, workspace_bytes, stream=0, batch=1,
     count = _int(0)
     _check(lib().strassen_autotune(ctypes.byref(req), ctypes.byref(best), log, log_capacity, ctypes.byref(count)))
     return best.as_dict(), [log[i].as_dict() for i in range(count.value)]
+
+
+def _ptr7(addresses):
+    if len(addresses) != 7:
+        raise ValueError("seven block addresses expected, got %d" % len(addresses))
+    return (_vp * 7)(*[int(a) for a in addresses])
+
+
+def strassen_bfs_form_shares(rows: int, h: int, A_share: int, lda: int, B_share: int, ldb: int, T_out, S_out, ld_out: int,
+                             stream: int = 0) -> None:
+    """T_out, S_out: seven device addresses each (block r of T_0..T_6 / S_0..S_6, rows x h)."""
+    _check(lib().strassen_bfs_form_shares(rows, h, A_share, lda, B_share, ldb, _ptr7(T_out), _ptr7(S_out), ld_out, stream))
+
+
+def strassen_bfs_combine_shares(rows: int, h: int, Q_in, ldq: int, C_share: int, ldc: int, stream: int = 0) -> None:
+    """Q_in: seven device addresses (block r of Q_0..Q_6, rows x h)."""
+    _check(lib().strassen_bfs_combine_shares(rows, h, _ptr7(Q_in), ldq, C_share, ldc, stream))
 
 
 def strassen_probe_fp64(kind: int, iters: int, stream: int = 0) -> float:
