@@ -374,6 +374,48 @@ def measure(name, steps, warmup, rank, world, dev, sampler_factory=None, want_cu
     return out, clocks, plan, (A, B, C)
 
 
+def run_bfs_step(args, rank, world, dev):
+    """One product over seven GPUs (strong scaling): every rank draws the same seeded A and B, keeps its share,
+    and the K timed steps are K whole distributed products; time = max over ranks."""
+    import torch
+    import torch.distributed as dist
+    from paper_1202_3173_b200 import caps, inputs
+    if world != caps.P:
+        raise SystemExit("--bfs-step needs exactly %d ranks (--gpus %d)" % (caps.P, caps.P))
+    n, cutoff, sched, batch, dist_name, seed, _ = WORKLOADS[args.workload]
+    if batch != 1 or n % 2:
+        raise SystemExit("--bfs-step takes a single product of even size")
+    A, B = inputs.pair(n, dist_name, seed, device=dev)
+    A_share, B_share = caps.take_share(A, rank), caps.take_share(B, rank)
+    del A, B
+    # the workload's top level is the distributed step; the levels below it run on each GPU
+    ops = caps.CudaOps(n // 2, dev, cutoff, None if sched == "auto" else sched[1:])
+    state, ex = caps.BfsStepRank(n, rank, ops), caps.TorchDistExchange()
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        caps.bfs_step(state, A_share, B_share, ex)
+    dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        caps.bfs_step(state, A_share, B_share, ex)
+    e1.record(stream)
+    dist.barrier()
+    torch.cuda.synchronize()
+    ms = reduce_max(e0.elapsed_time(e1) / args.steps, dev)
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": 2.0 * n ** 3 / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": describe(args.workload), "parallelism": "one BFS step over 7 GPUs (Algorithm 2, k = 1)",
+                       "sub_problem": {"n": n // 2, "schedule": ops.plan.schedule, "levels": ops.plan.level_sizes},
+                       "message_words": n * n // (4 * caps.P), "all_to_alls_per_step": 3},
+            "gpu_launches": args.steps * (ops.plan.launch_count + 2)}), flush=True)
+    ops.close()
+
+
 def run_reference(args, rank, world):
     """The reference arm: the CPU oracle as it stands, on the host cores, rank 0 only."""
     if rank != 0:
@@ -416,6 +458,10 @@ def main():
     ap.add_argument("--no-autotune", action="store_true", help="skip the measured choice of steps and interleaving")
     ap.add_argument("--no-per-config", action="store_true", help="skip the short measurement of the other configurations")
     ap.add_argument("--graph", action="store_true", help="also time the plan replayed as one CUDA graph")
+    ap.add_argument("--bfs-step", action="store_true",
+                    help="with --gpus 7: time ONE product spread over the seven GPUs as a BFS step of CAPS (Algorithm 2, "
+                         "k = 1: local sums, three all-to-alls over NCCL, the n/2 sub-products on the single-GPU path, local "
+                         "combine) instead of seven independent replicas")
     ap.add_argument("--check-launch", action="store_true",
                     help="no GPU work: every rank joins a gloo group and exchanges a stand-in time through the same reduction "
                          "(checks the launcher plumbing of --gpus N on a machine without GPUs)")
@@ -468,6 +514,12 @@ def main():
     if world > 1:
         dist.barrier()
     from paper_1202_3173_b200 import Plan, binding
+
+    if args.bfs_step:
+        run_bfs_step(args, rank, world, dev)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     n, cutoff, sched, batch, dist_name, seed, _ = WORKLOADS[args.workload]
     head, clocks, plan, (A, B, C) = measure(args.workload, args.steps, args.warmup, rank, world, dev,
