@@ -64,7 +64,8 @@ typedef enum strassen_kernel_kind {
     STRASSEN_K_PEEL = 5,       /* peeling fix-ups: rank-one update, last column, last row           */
     STRASSEN_K_SCALE = 6,      /* diagonal scaling passes (STRASSEN_FLAG_SCALE_*)                   */
     STRASSEN_K_FUSED_STEP = 7, /* a whole BFS step of the deepest level (sums, products, U-chain) in one kernel */
-    STRASSEN_K_COUNT = 8
+    STRASSEN_K_LINCOMB = 8,    /* generic bilinear schemes: linear combinations of blocks / of products       */
+    STRASSEN_K_COUNT = 9
 } strassen_kernel_kind;
 
 /* Extended plan description.  Zero-initialise, then set what differs from the default. */
@@ -279,6 +280,40 @@ typedef struct strassen_tune_entry {
 
 int strassen_autotune(const strassen_tune_request *request, strassen_tune_entry *best, strassen_tune_entry *log,
                       int log_capacity, int *log_count);
+
+/*
+ * Other bilinear schemes through the same traversal [Section 6.6 "Parallelizing other algorithms": every fast
+ * square matrix multiplication multiplies n0 x n0 block matrices with q < n0^3 products of linear combinations
+ * of the blocks; "the BFS and DFS determine whether the q multiplications are performed in parallel or
+ * sequentially"; the recursive classical algorithm is the case q = n0^3].
+ *
+ * A scheme is three tables of small integers (blocks numbered row-major, b = n0 * block_row + block_column):
+ *   u, v   q x n0^2:   T_j = sum_b u[j][b] A_b,   S_j = sum_b v[j][b] B_b,   Q_j = T_j . S_j
+ *   w      n0^2 x q:   C_b = sum_j w[b][j] Q_j
+ * strassen_scheme_check verifies on the host that the tables multiply matrices (the coefficient of
+ * A_(a,b) B_(c,d) in C_(e,f) is 1 where b = c, a = e, d = f and 0 elsewhere); plan creation runs the same check.
+ * Built-in names: "classical" (<2,2,2;8>), "strassen" (<2,2,2;7>, the original form with 18 additions),
+ * "winograd" (<2,2,2;7>, Appendix A with its shared sub-sums written out).
+ *
+ * The plan is an ordinary strassen_plan (strassen_dgemm, strassen_dgemm_host, workspace and query calls, destroy).
+ * Level rule: m_0 = n, m_{i+1} = m_i / n0 while m_i > cutoff, and every m_i that is split must be divisible by
+ * n0 -- generic schemes do not peel (STRASSEN_INVALID_ARG otherwise).  opt->schedule: one 'B' (all q sub-products
+ * of a step side by side, batched) or 'D' (one after another, one triple of workspace) per level, or NULL /
+ * "auto" for the Limited-Memory rule [Section 3.4].  Combinations that are a single block with coefficient 1 are
+ * used in place.  Of opt->flags only CUDA_GRAPH and HOST_PIPELINE apply.  Every linear combination is one
+ * streaming launch (each term read once per output element), the products run on the batched FP64 GEMM.
+ */
+typedef struct strassen_scheme {
+    int n0;             /* blocks per side, 2 .. 4                                                   */
+    int q;              /* products per step, 1 .. 64                                                */
+    const int8_t *u;    /* q x n0^2, row-major, host memory, read during the call only               */
+    const int8_t *v;    /* q x n0^2                                                                  */
+    const int8_t *w;    /* n0^2 x q                                                                  */
+} strassen_scheme;
+
+int strassen_scheme_check(const strassen_scheme *scheme);
+strassen_plan *strassen_plan_create_scheme(const strassen_options *opt, const strassen_scheme *scheme);
+strassen_plan *strassen_plan_create_named_scheme(const strassen_options *opt, const char *name);
 
 /*
  * The two local steps of ONE BFS step spread over seven GPUs [Algorithm 2, BFS(A, B, C, k) with k = 1:

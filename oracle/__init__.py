@@ -18,6 +18,9 @@ paper that needs no matrix data:
   (a BFS step stores 7 triples S_j,T_j,Q_j of quarter size, a DFS step one),
   ``mem_um_closed_form`` -- Mem_UM = 7 n^2 / P^{2/w0} - 4 n^2 / P at P = 7^k.
 * ``effective_gflops`` -- 2 n^3 / (t 10^9) (Section 5.2).
+* ``bilinear_product``, ``brent_residual``, ``classical_scheme`` -- the recursion
+  for any <n0, n0, n0; q> bilinear scheme (Section 6.6) on numpy blocks, the
+  identities its tables must satisfy, and the table of the classical algorithm.
 * ``bfs_row_blocks``, ``bfs_share``, ``bfs_unshare``, ``bfs_form_shares``,
   ``bfs_combine_shares`` -- one BFS step spread over seven processors
   (Algorithm 2 with k = 1; layout of Section 3.2) restated on numpy blocks.
@@ -319,3 +322,61 @@ def bfs_combine_shares(Q):
     u2 = u1 + q[4]
     u3 = u1 + q[2]
     return np.vstack((np.hstack((q[0] + q[1], u3 + q[5])), np.hstack((u2 - q[6], u2 + q[2]))))
+
+
+# ---- any <n0, n0, n0; q> bilinear scheme (Section 6.6 "Parallelizing other algorithms") -------------------
+# u, v: q x n0^2, w: n0^2 x q (blocks row-major):  T_j = sum_b u[j][b] A_b,  S_j = sum_b v[j][b] B_b,
+# Q_j = T_j . S_j,  C_b = sum_j w[b][j] Q_j.
+
+def brent_residual(n0, q, u, v, w):
+    """Largest violation of the identities that make the tables a matrix multiplication: the coefficient of
+    A_(a,b) B_(c,d) in C_(e,f) is 1 where b = c, a = e, d = f, and 0 elsewhere.  0 for a correct scheme."""
+    u, v, w = np.asarray(u, dtype=np.int64), np.asarray(v, dtype=np.int64), np.asarray(w, dtype=np.int64)
+    got = np.einsum("jx,jy,zj->xyz", u, v, w)
+    want = np.zeros_like(got)
+    for a in range(n0):
+        for b in range(n0):
+            for d in range(n0):
+                want[a * n0 + b, b * n0 + d, a * n0 + d] = 1
+    return int(np.abs(got - want).max())
+
+
+def classical_scheme(n0: int):
+    """The classical algorithm as a <n0, n0, n0; n0^3> scheme: product (i, k, j) is A_(i,k) B_(k,j), added to C_(i,j)."""
+    q = n0 ** 3
+    u, v, w = np.zeros((q, n0 * n0), dtype=int), np.zeros((q, n0 * n0), dtype=int), np.zeros((n0 * n0, q), dtype=int)
+    t = 0
+    for i in range(n0):
+        for j in range(n0):
+            for k in range(n0):
+                u[t, i * n0 + k] = 1
+                v[t, k * n0 + j] = 1
+                w[i * n0 + j, t] = 1
+                t += 1
+    return n0, q, u.tolist(), v.tolist(), w.tolist()
+
+
+def bilinear_product(A, B, scheme, cutoff: int):
+    """C = A.B by the recursion of the scheme down to sizes <= cutoff, then the classical oracle.
+    Returns (C, number of base products)."""
+    n0, q, u, v, w = scheme
+    u, v, w = np.asarray(u), np.asarray(v), np.asarray(w)
+    A, B = np.asarray(A, dtype=np.float64), np.asarray(B, dtype=np.float64)
+    m = A.shape[0]
+    if m <= cutoff:
+        return classical(A, B), 1
+    if m % n0:
+        raise ValueError("size %d is not divisible by n0 = %d" % (m, n0))
+    hh = m // n0
+    blk = lambda X, b: X[(b // n0) * hh:(b // n0 + 1) * hh, (b % n0) * hh:(b % n0 + 1) * hh]
+    Q, calls = [], 0
+    for j in range(q):
+        T = sum(int(u[j, b]) * blk(A, b) for b in range(n0 * n0) if u[j, b])
+        S = sum(int(v[j, b]) * blk(B, b) for b in range(n0 * n0) if v[j, b])
+        Qj, c = bilinear_product(np.ascontiguousarray(T), np.ascontiguousarray(S), scheme, cutoff)
+        Q.append(Qj)
+        calls += c
+    C = np.empty((m, m))
+    for b in range(n0 * n0):
+        blk(C, b)[...] = sum(int(w[b, j]) * Q[j] for j in range(q) if w[b, j])
+    return C, calls

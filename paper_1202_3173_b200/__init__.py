@@ -23,10 +23,24 @@ class Plan:
     """
 
     def __init__(self, n, cutoff=0, schedule=None, batch=1, workspace_budget_bytes=0, lda=0, ldb=0, ldc=0,
-                 stride_a=0, stride_b=0, stride_c=0, flags=0):
+                 stride_a=0, stride_b=0, stride_c=0, flags=0, scheme=None):
+        """``scheme``: None for the Strassen-Winograd step of the paper's Appendix A; the name of a built-in
+        bilinear scheme ("classical", "strassen", "winograd"); or a tuple (n0, q, u, v, w) of coefficient tables
+        for any <n0, n0, n0; q> scheme (Section 6.6) -- sizes must then divide by n0 at every level."""
         self.n, self.cutoff, self.batch = int(n), int(cutoff), int(batch)
-        self._h = binding.strassen_plan_create_ex(n, cutoff, schedule, batch, lda, ldb, ldc, stride_a, stride_b,
-                                                  stride_c, workspace_budget_bytes, flags)
+        if scheme is None:
+            self._h = binding.strassen_plan_create_ex(n, cutoff, schedule, batch, lda, ldb, ldc, stride_a, stride_b,
+                                                      stride_c, workspace_budget_bytes, flags)
+        else:
+            if lda or ldb or ldc or stride_a or stride_b or stride_c:
+                raise ValueError("plans for a generic scheme take packed matrices")
+            if isinstance(scheme, str):
+                self._h = binding.strassen_plan_create_named_scheme(n, cutoff, schedule, scheme, batch,
+                                                                    workspace_budget_bytes, flags)
+            else:
+                n0, q, u, v, w = scheme
+                self._h = binding.strassen_plan_create_scheme(n, cutoff, schedule, n0, q, u, v, w, batch,
+                                                              workspace_budget_bytes, flags)
         self._ws = None
         self._packed = not (lda or ldb or ldc or stride_a or stride_b or stride_c)
         self._want = (self.n, self.n) if self.batch == 1 else (self.batch, self.n, self.n)

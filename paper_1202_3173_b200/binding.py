@@ -24,8 +24,8 @@ STRASSEN_FLAG_NO_FUSED_STEP = 128
 STRASSEN_FLAG_NO_DFS_FOLD = 256
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SCHEDULE", -3: "WORKSPACE_TOO_SMALL", -4: "ALIAS",
                 -5: "MISALIGNED", -6: "CUDA_ERROR", -7: "OUT_OF_MEMORY"}
-K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_SCALE, K_FUSED_STEP, K_COUNT = range(9)
-KERNEL_KINDS = ("form", "gemm", "recombine", "form_one", "accumulate", "peel", "scale", "fused_step")
+K_FORM, K_GEMM, K_RECOMBINE, K_FORM_ONE, K_ACCUMULATE, K_PEEL, K_SCALE, K_FUSED_STEP, K_LINCOMB, K_COUNT = range(10)
+KERNEL_KINDS = ("form", "gemm", "recombine", "form_one", "accumulate", "peel", "scale", "fused_step", "lincomb")
 
 # every symbol the header declares: (name, restype, argtypes)
 _vp, _i64, _sz, _cp, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_char_p, ctypes.c_int
@@ -37,6 +37,11 @@ class strassen_options(ctypes.Structure):
                 ("lda", _i64), ("ldb", _i64), ("ldc", _i64),
                 ("stride_a", _i64), ("stride_b", _i64), ("stride_c", _i64),
                 ("workspace_budget_bytes", _sz), ("flags", _i64)]
+
+
+class strassen_scheme(ctypes.Structure):
+    _fields_ = [("n0", _int), ("q", _int), ("u", ctypes.POINTER(ctypes.c_int8)), ("v", ctypes.POINTER(ctypes.c_int8)),
+                ("w", ctypes.POINTER(ctypes.c_int8))]
 
 
 class strassen_tune_request(ctypes.Structure):
@@ -76,6 +81,9 @@ SYMBOLS = [
     ("strassen_autotune", _int, [ctypes.POINTER(strassen_tune_request), ctypes.POINTER(strassen_tune_entry),
                                  ctypes.POINTER(strassen_tune_entry), _int, ctypes.POINTER(_int)]),
     ("strassen_probe_fp64", _int, [_int, _i64, _vp, _dp]),
+    ("strassen_scheme_check", _int, [ctypes.POINTER(strassen_scheme)]),
+    ("strassen_plan_create_scheme", _vp, [ctypes.POINTER(strassen_options), ctypes.POINTER(strassen_scheme)]),
+    ("strassen_plan_create_named_scheme", _vp, [ctypes.POINTER(strassen_options), _cp]),
     ("strassen_bfs_form_shares", _int, [_i64, _i64, _vp, _i64, _vp, _i64, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i64, _vp]),
     ("strassen_bfs_combine_shares", _int, [_i64, _i64, ctypes.POINTER(_vp), _i64, _vp, _i64, _vp]),
     ("strassen_dgemm_static", _int, [_i64, _vp, _vp, _vp, _vp]),
@@ -227,6 +235,39 @@ def strassen_autotune(n, A, B, C, workspace, workspace_bytes, stream=0, batch=1,
     count = _int(0)
     _check(lib().strassen_autotune(ctypes.byref(req), ctypes.byref(best), log, log_capacity, ctypes.byref(count)))
     return best.as_dict(), [log[i].as_dict() for i in range(count.value)]
+
+
+def _scheme(n0, q, u, v, w):
+    """(struct, keep-alive) for tables given as nested sequences: u, v are q x n0^2, w is n0^2 x q."""
+    def flat(t, rows, cols):
+        cells = [int(x) for row in t for x in row]
+        if len(t) != rows or len(cells) != rows * cols:
+            raise ValueError("a %d x %d table is expected" % (rows, cols))
+        return (ctypes.c_int8 * len(cells))(*cells)
+    bu, bv, bw = flat(u, q, n0 * n0), flat(v, q, n0 * n0), flat(w, n0 * n0, q)
+    return strassen_scheme(n0, q, bu, bv, bw), (bu, bv, bw)
+
+
+def strassen_scheme_check(n0, q, u, v, w) -> None:
+    s, keep = _scheme(n0, q, u, v, w)
+    _check(lib().strassen_scheme_check(ctypes.byref(s)))
+
+
+def strassen_plan_create_scheme(n, cutoff, schedule, n0, q, u, v, w, batch=1, workspace_budget_bytes=0, flags=0) -> int:
+    o = strassen_options(n, cutoff, _sched(schedule), batch, 0, 0, 0, 0, 0, 0, workspace_budget_bytes, flags)
+    s, keep = _scheme(n0, q, u, v, w)
+    h = lib().strassen_plan_create_scheme(ctypes.byref(o), ctypes.byref(s))
+    if not h:
+        raise StrassenError(-1, strassen_last_error())
+    return h
+
+
+def strassen_plan_create_named_scheme(n, cutoff, schedule, name, batch=1, workspace_budget_bytes=0, flags=0) -> int:
+    o = strassen_options(n, cutoff, _sched(schedule), batch, 0, 0, 0, 0, 0, 0, workspace_budget_bytes, flags)
+    h = lib().strassen_plan_create_named_scheme(ctypes.byref(o), name.encode())
+    if not h:
+        raise StrassenError(-1, strassen_last_error())
+    return h
 
 
 def _ptr7(addresses):

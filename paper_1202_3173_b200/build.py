@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libstrassen_b200.so")
-SOURCES = ["plan.cpp", "add_kernels.cu", "add3_kernels.cu", "gemm_f64.cu", "fused_step.cu", "bfs_shares.cu", "probe.cu", "api.cu", "static_entry.cu", "tune.cu", "scale_kernels.cu"]
+SOURCES = ["plan.cpp", "add_kernels.cu", "add3_kernels.cu", "gemm_f64.cu", "fused_step.cu", "bfs_shares.cu", "bilinear.cu", "bilinear_plan.cpp", "probe.cu", "api.cu", "static_entry.cu", "tune.cu", "scale_kernels.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -593,6 +593,7 @@ int launches_of(const Launch &op)
     case OP_FORM3: return chunks(op.count * 2);
     case OP_RECOMBINE3: return chunks(op.count);
     case OP_FUSED_STEP: return chunks(op.count);
+    case OP_LINCOMB: return chunks(op.count);
     }
     return 0;
 }

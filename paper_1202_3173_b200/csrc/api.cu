@@ -8,6 +8,7 @@
 #include <string>
 #include <vector>
 
+#include "bilinear.h"
 #include "kernels.h"
 #include "plan.h"
 
@@ -56,6 +57,7 @@ struct strassen_plan {
     cudaStream_t capture_stream = nullptr;
     cudaGraphExec_t graph_exec = nullptr;
     const void *graph_ptrs[4] = {nullptr, nullptr, nullptr, nullptr};   // A, B, C, workspace the graph was captured for
+    bool scheme_vec = false;              // generic bilinear plan: every level size, leading dimension and stride is even
     double acc_ms[STRASSEN_K_COUNT] = {};
     int64_t launches[STRASSEN_K_COUNT] = {};
     int64_t launch_total = 0;
@@ -70,6 +72,7 @@ int family(int op_kind)
     if (op_kind == OP_RECOMBINE2 || op_kind == OP_RECOMBINE3) return STRASSEN_K_RECOMBINE;
     if (op_kind == OP_SCALE_IN || op_kind == OP_SCALE_OUT) return STRASSEN_K_SCALE;
     if (op_kind == OP_FUSED_STEP) return STRASSEN_K_FUSED_STEP;
+    if (op_kind == OP_LINCOMB) return STRASSEN_K_LINCOMB;
     return op_kind;
 }
 
@@ -203,6 +206,12 @@ int enqueue_launches(strassen_plan *p, const Bases &bases, bool bases16, cudaStr
         case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
         case OP_FORM3: e = launch_form3(p->d_tab, op, bases, stream, &launched); break;
         case OP_RECOMBINE3: e = launch_recombine3(p->d_tab, op, bases, stream, &launched); break;
+        case OP_LINCOMB: {
+            // the linear combinations of a generic scheme take 16-byte accesses where the whole plan allows them
+            const LinComb &lc = reinterpret_cast<const LinComb *>(p->d.lincombs.data())[op.j];
+            e = launch_lincomb(p->d_tab, op, lc, bases, bases16 && p->scheme_vec, stream, &launched);
+            break;
+        }
         case OP_FUSED_STEP: e = launch_fused_step(p->d_tab, op, bases, p->sm_count, stream, &launched); break;
         case OP_SCALE_IN: e = launch_scale_in(p->d, bases, stream, &launched); break;
         case OP_SCALE_OUT: e = launch_scale_out(p->d, bases, stream, &launched); break;
@@ -379,6 +388,94 @@ strassen_plan *create(const strassen_options &o)
     return p;
 }
 
+// A plan for a generic <n0, n0, n0; q> scheme: the same handle type, its own level rule (sizes divide by n0, no
+// peeling) and launch list.
+strassen_plan *create_scheme(const strassen_options &o, const Scheme &s)
+{
+    g_error.clear();
+    const std::string bad = validate_scheme(s);
+    if (!bad.empty()) {
+        fail(STRASSEN_INVALID_ARG, "not a matrix-multiplication scheme: " + bad);
+        return nullptr;
+    }
+    const int64_t n = o.n, batch = o.batch == 0 ? 1 : o.batch;
+    if (n < 1 || o.cutoff < 1 || batch < 1 || n > (int64_t(1) << 30)) {
+        fail(STRASSEN_INVALID_ARG, "n, cutoff and batch must be positive (n at most 2^30)");
+        return nullptr;
+    }
+    if (o.flags & ~int64_t(STRASSEN_FLAG_CUDA_GRAPH | STRASSEN_FLAG_HOST_PIPELINE)) {
+        fail(STRASSEN_INVALID_ARG, "generic schemes take only the CUDA_GRAPH and HOST_PIPELINE flags");
+        return nullptr;
+    }
+    strassen_plan *p = new (std::nothrow) strassen_plan;
+    if (!p) {
+        fail(STRASSEN_OUT_OF_MEMORY, "out of host memory");
+        return nullptr;
+    }
+    PlanDesc &d = p->d;
+    d.n = n; d.cutoff = o.cutoff; d.batch = batch;
+    d.lda = o.lda ? o.lda : n; d.ldb = o.ldb ? o.ldb : n; d.ldc = o.ldc ? o.ldc : n;
+    d.stride_a = o.stride_a ? o.stride_a : d.lda * n;
+    d.stride_b = o.stride_b ? o.stride_b : d.ldb * n;
+    d.stride_c = o.stride_c ? o.stride_c : d.ldc * n;
+    const int64_t ldmax = 0x7fffffff;
+    auto bail = [&](int status, const std::string &msg) {
+        fail(status, msg);
+        delete p;
+        return static_cast<strassen_plan *>(nullptr);
+    };
+    if (d.lda < n || d.ldb < n || d.ldc < n || d.lda > ldmax || d.ldb > ldmax || d.ldc > ldmax)
+        return bail(STRASSEN_INVALID_ARG, "leading dimensions must be >= n and fit 31 bits");
+    if (d.stride_a < 0 || d.stride_b < 0 || (batch > 1 && d.stride_c < (n - 1) * d.ldc + n))
+        return bail(STRASSEN_INVALID_ARG, "batch members of C must not overlap; strides must be non-negative");
+    d.sizes = scheme_level_sizes(n, o.cutoff, s.n0);
+    if (d.sizes.empty())
+        return bail(STRASSEN_INVALID_ARG, "a generic scheme needs every level size above the cutoff to be divisible by n0 (no peeling)");
+    d.cutoff = d.sizes.back();
+    const size_t L = d.sizes.size() - 1;
+    const bool want_auto = !o.schedule || strcmp(o.schedule, "auto") == 0;
+    if (want_auto) {
+        size_t budget = o.workspace_budget_bytes;
+        if (budget == 0 && L > 0) {
+            size_t free_b = 0, total_b = 0;
+            if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) {
+                cudaGetLastError();
+                return bail(STRASSEN_CUDA_ERROR, "schedule \"auto\" without a workspace budget needs a CUDA device");
+            }
+            budget = free_b > (size_t(1) << 30) ? free_b - (size_t(1) << 30) : 0;
+        }
+        bool found = false;       // Limited-Memory rule: the fewest leading DFS steps, then BFS steps only
+        for (size_t ell = 0; ell <= L && !found; ++ell) {
+            const std::string sched = std::string(ell, 'D') + std::string(L - ell, 'B');
+            const int64_t w = scheme_workspace_words(s, d.sizes, sched, batch);
+            if (w >= 0 && size_t(w) <= budget / 8) {
+                d.schedule = sched;
+                found = true;
+            }
+        }
+        if (!found) return bail(STRASSEN_WORKSPACE_TOO_SMALL, "even the all-DFS schedule does not fit the workspace budget");
+    } else {
+        d.schedule = o.schedule;
+        if (d.schedule.size() != L) return bail(STRASSEN_BAD_SCHEDULE, "the schedule must have one character per level");
+        for (char c : d.schedule)
+            if (c != 'B' && c != 'D') return bail(STRASSEN_BAD_SCHEDULE, "schedule characters must be 'B' or 'D'");
+        if (o.workspace_budget_bytes && size_t(scheme_workspace_words(s, d.sizes, d.schedule, batch)) * 8 > o.workspace_budget_bytes)
+            return bail(STRASSEN_WORKSPACE_TOO_SMALL, "the schedule needs more workspace than the budget allows");
+    }
+    const std::string err = build_scheme_plan(&d, s);
+    if (!err.empty()) return bail(STRASSEN_INVALID_ARG, err);
+    p->use_graph = (o.flags & STRASSEN_FLAG_CUDA_GRAPH) != 0;
+    p->host_pipeline = (o.flags & STRASSEN_FLAG_HOST_PIPELINE) != 0;
+    p->scheme_vec = ((d.lda | d.ldb | d.ldc | d.stride_a | d.stride_b | d.stride_c) & 1) == 0;
+    for (size_t i = 0; i < d.sizes.size(); ++i) p->scheme_vec = p->scheme_vec && (i == 0 || d.sizes[i] % 2 == 0);
+    for (const Launch &op : d.launches) {
+        const int k = launches_of(op);
+        p->launches[family(op.kind)] += k;
+        p->launch_total += k;
+    }
+    return p;
+}
+
 }  // namespace
 
 namespace strassen {
@@ -402,6 +499,52 @@ strassen_plan *strassen_plan_create_ex(const strassen_options *opt)
         return nullptr;
     }
     return create(*opt);
+}
+
+strassen_plan *strassen_plan_create_scheme(const strassen_options *opt, const strassen_scheme *scheme)
+{
+    if (!opt || !scheme || !scheme->u || !scheme->v || !scheme->w) {
+        fail(STRASSEN_INVALID_ARG, "options, scheme and its three tables must be non-NULL");
+        return nullptr;
+    }
+    if (scheme->n0 < 2 || scheme->n0 > 4 || scheme->q < 1 || scheme->q > kMaxSchemeProducts) {
+        fail(STRASSEN_INVALID_ARG, "a scheme needs 2 <= n0 <= 4 and 1 <= q <= 64");
+        return nullptr;
+    }
+    Scheme s;
+    s.n0 = scheme->n0; s.q = scheme->q;
+    const size_t cells = size_t(s.q) * s.n0 * s.n0;
+    s.u.assign(scheme->u, scheme->u + cells);
+    s.v.assign(scheme->v, scheme->v + cells);
+    s.w.assign(scheme->w, scheme->w + cells);
+    return create_scheme(*opt, s);
+}
+
+strassen_plan *strassen_plan_create_named_scheme(const strassen_options *opt, const char *name)
+{
+    Scheme s;
+    if (!opt || !name || !builtin_scheme(name, &s)) {
+        fail(STRASSEN_INVALID_ARG, "options must be non-NULL and the name one of \"classical\", \"strassen\", \"winograd\"");
+        return nullptr;
+    }
+    return create_scheme(*opt, s);
+}
+
+int strassen_scheme_check(const strassen_scheme *scheme)
+{
+    g_error.clear();
+    if (!scheme || !scheme->u || !scheme->v || !scheme->w) return fail(STRASSEN_INVALID_ARG, "scheme and its three tables must be non-NULL");
+    if (scheme->n0 < 2 || scheme->n0 > 4 || scheme->q < 1 || scheme->q > kMaxSchemeProducts)
+        return fail(STRASSEN_INVALID_ARG, "a scheme needs 2 <= n0 <= 4 and 1 <= q <= 64");
+    Scheme s;
+    s.n0 = scheme->n0; s.q = scheme->q;
+    const size_t cells = size_t(s.q) * s.n0 * s.n0;
+    s.u.assign(scheme->u, scheme->u + cells);
+    s.v.assign(scheme->v, scheme->v + cells);
+    s.w.assign(scheme->w, scheme->w + cells);
+    const std::string bad = validate_scheme(s);
+    if (!bad.empty()) return fail(STRASSEN_INVALID_ARG, bad);
+    return STRASSEN_OK;
 }
 
 int strassen_dgemm(strassen_plan *p, const double *A, const double *B, double *C, void *stream_v)
@@ -594,13 +737,13 @@ int64_t strassen_plan_launches_of(const strassen_plan *p, int kind)
 
 double strassen_plan_pass_bytes(const strassen_plan *p)
 {
-    if (!p) return -1.0;
+    if (!p || p->d.scheme_n0) return -1.0;       // the model describes the Strassen-Winograd plans only
     return plan_model_parts(p->d.sizes, p->d.schedule, p->d.batch, p->d.fused_step).pass_bytes;
 }
 
 double strassen_plan_model_ms(const strassen_plan *p)
 {
-    if (!p) return -1.0;
+    if (!p || p->d.scheme_n0) return -1.0;
     return plan_model_ms(p->d.sizes, p->d.schedule, p->d.batch, p->d.fused_step);
 }
 

@@ -137,6 +137,11 @@ inline bool fused_step_pays(int64_t h, int64_t parents, int sms)
     return tiles < sms;
 }
 
+// Generic bilinear schemes (bilinear.cu): one linear-combination launch over op.count parents.
+struct LinComb;
+cudaError_t launch_lincomb(const Node *tab, const Launch &op, const LinComb &lc, const Bases &bases, bool vec, cudaStream_t stream,
+                           int *launched);
+
 constexpr int kNominalSMs = 148;   // B200; used where launches are counted without a device at hand
 
 // Sets the shared-memory attribute of every GEMM kernel shape on the current device (idempotent).

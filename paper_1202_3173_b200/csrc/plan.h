@@ -39,7 +39,8 @@ enum OpKind : int32_t {
     OP_SCALE_OUT = 9,  // diagonal scaling: C scaled back in place
     OP_FORM3 = 10,     // three BFS levels at once: sums of the children, grandchildren and great-grandchildren
     OP_RECOMBINE3 = 11, // three BFS levels at once: 343 great-grandchild products -> the parent's C
-    OP_FUSED_STEP = 12  // a whole BFS step of the deepest level in one kernel: quadrants of A, B -> C
+    OP_FUSED_STEP = 12, // a whole BFS step of the deepest level in one kernel: quadrants of A, B -> C
+    OP_LINCOMB = 13     // generic bilinear scheme: one output matrix per parent as a linear combination (j = index of its LinComb)
 };
 
 // Regular layout of the workspace regions a two- or three-level launch writes / reads (element offsets
@@ -109,6 +110,8 @@ struct PlanDesc {
     int64_t ws_words = 0;           // total workspace words
     std::vector<Node> nodes;        // all node tables, concatenated
     std::vector<Launch> launches;   // replayed in order by strassen_dgemm
+    std::vector<unsigned char> lincombs;   // generic bilinear schemes: the LinComb records OP_LINCOMB launches refer to (bilinear.h)
+    int scheme_n0 = 0, scheme_q = 0;       // ... and the scheme's shape (0: the Strassen-Winograd plan of Appendix A)
 };
 
 // How many levels, starting at `level`, one pass forms and recombines (1 .. max_fused) under schedule

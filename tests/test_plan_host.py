@@ -167,17 +167,17 @@ def test_launch_lists():
     single = binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES
     p = Plan(4096, 512, "BBB", flags=single)
     # (343 x 16 tiles = 37 full rounds of 148 + 12: the leaf owning the leftover runs as a second, small-tile launch)
-    assert p.launches_by_kind() == {"form": 3, "gemm": 2, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 0}
+    assert p.launches_by_kind() == {"form": 3, "gemm": 2, "recombine": 3, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 0, "lincomb": 0}
     assert p.launch_count == 8
     p.close()
     # default: up to three BFS levels share one formation pass and one recombination pass
     p = Plan(4096, 512, "BBB")
-    assert p.launches_by_kind() == {"form": 1, "gemm": 2, "recombine": 1, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 0}
+    assert p.launches_by_kind() == {"form": 1, "gemm": 2, "recombine": 1, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 0, "lincomb": 0}
     p.close()
     # at most two levels per pass: the two deepest levels pair up
     two = binding.STRASSEN_FLAG_TWO_LEVEL_PASSES
     p = Plan(4096, 512, "BBB", flags=two)
-    assert p.launches_by_kind() == {"form": 2, "gemm": 2, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 0}
+    assert p.launches_by_kind() == {"form": 2, "gemm": 2, "recombine": 2, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 0, "lincomb": 0}
     p.close()
     # DFS on top: 7 x (form_one [not for j = 0, 1], sub-tree, accumulate)
     p = Plan(16384, 512, "DBBBB", flags=single)
@@ -229,7 +229,7 @@ def test_launch_lists():
     # a deepest BFS step whose products would leave most SMs idle runs as one fused kernel (no sums, no products in memory)
     p = Plan(512, 256, "B")
     assert p.launches_by_kind() == {"form": 0, "gemm": 0, "recombine": 0, "form_one": 0, "accumulate": 0, "peel": 0,
-                                    "scale": 0, "fused_step": 1}
+                                    "scale": 0, "fused_step": 1, "lincomb": 0}
     assert p.base_products == 7
     p.close()
     p = Plan(512, 256, "B", flags=binding.STRASSEN_FLAG_NO_FUSED_STEP)
@@ -238,7 +238,7 @@ def test_launch_lists():
     p.close()
     p = Plan(4096, 512, "BBB", flags=binding.STRASSEN_FLAG_FUSED_STEP)     # forced: a two-level pass above the fused deepest step
     k = p.launches_by_kind()
-    assert k == {"form": 1, "gemm": 0, "recombine": 1, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 1}
+    assert k == {"form": 1, "gemm": 0, "recombine": 1, "form_one": 0, "accumulate": 0, "peel": 0, "scale": 0, "fused_step": 1, "lincomb": 0}
     assert p.base_products == 343
     p.close()
     p = Plan(1025, 512, "D", flags=binding.STRASSEN_FLAG_FUSED_STEP)       # only a BFS step can be fused
