@@ -380,7 +380,7 @@ cudaError_t configure_fused_step_kernels()
     return e;
 }
 
-bool fused_step_uses_wide_tiles(int64_t h, int64_t count, int sms)
+static bool fused_step_uses_wide_tiles(int64_t h, int64_t count, int sms)
 {
     // the wide tile moves half the operand bytes per flop; it needs enough tiles to keep every SM busy
     const int64_t wide_tiles = ((h + FWide::TM - 1) / FWide::TM) * ((h + FWide::TN - 1) / FWide::TN) * count;

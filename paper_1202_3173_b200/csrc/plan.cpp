@@ -253,7 +253,6 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
     const int L = int(sched.size());
     ModelParts out{};
     double visits = double(batch), sequential = 1.0;   // node visits at the current level; sub-trees run one after another
-    int64_t parents_exact = batch;
     const bool fused = L > 0 && fused_step_chosen(fused_mode, sched, sizes[L], [&] {
         int64_t live = batch;
         for (int i = 0; i + 1 < L; ++i)
@@ -286,10 +285,7 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         const double words = g == 1 ? 27.0 : g == 2 ? 28.0 + 16.25 : 49.0 + 25.5;    // per parent, in h^2 of its children
         out.pass_bytes += visits * words * h * h * 8.0;
         out.launches += 2.0 * sequential;
-        for (int i = 0; i < g; ++i) {
-            visits *= 7.0;
-            parents_exact *= 7;
-        }
+        for (int i = 0; i < g; ++i) visits *= 7.0;
         level += g;
     }
     if (fused) {
@@ -329,7 +325,6 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         out.thin_bytes += leaves * 2.0 * double(b) * double(b) * 8.0;
         out.launches += 2.0 * sequential;
     }
-    (void)parents_exact;
     return out;
 }
 

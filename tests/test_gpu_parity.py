@@ -354,7 +354,8 @@ def test_errors_on_device():
     plan.close()
 
 
-@pytest.mark.parametrize("n,cutoff,sched,flags", [(2048, 16, "BBBBBBB", 0), (2048, 16, "BBBBBBB", 1), (1024, 8, "BBBBBBB", 32)])
+@pytest.mark.parametrize("n,cutoff,sched,flags", [(2048, 16, "BBBBBBB", 0), (2048, 16, "BBBBBBB", 1), (1024, 8, "BBBBBBB", 32),
+                                                  (2048, 16, "BBBBBBB", 64)])      # 64: 117 649 parents through the fused step
 def test_item_lists_longer_than_one_launch_covers(n, cutoff, sched, flags):
     # 7^6 = 117 649 parents at the deepest level and 7^7 = 823 543 leaves: the streaming kernels and the thin
     # products (8 x 8 leaves are all remainder) cut their item lists into launches of at most 32 768 items
