@@ -139,7 +139,11 @@ def test_random_sizes_cutoffs_and_schedules():
         L = len(oracle.level_sizes(n, cutoff)) - 1
         sched = "".join(rng.choice(list("BD"), size=L))
         batch = int(rng.integers(1, 4))
-        check_full(n, cutoff, sched, "int8", 9000 + case, batch=batch)
+        # alternate between the default plan (small deepest BFS steps run fused), the three-launch form of every step,
+        # and separate fold passes in every DFS step
+        flags = (0, binding.STRASSEN_FLAG_NO_FUSED_STEP, binding.STRASSEN_FLAG_NO_FUSED_STEP | binding.STRASSEN_FLAG_NO_DFS_FOLD,
+                 binding.STRASSEN_FLAG_FUSED_STEP)[case % 4]
+        check_full(n, cutoff, sched, "int8", 9000 + case, batch=batch, flags=flags)
 
 
 def test_pointers_that_are_only_8_byte_aligned():
@@ -238,7 +242,8 @@ FUSED, UNFUSED = binding.STRASSEN_FLAG_FUSED_STEP, binding.STRASSEN_FLAG_NO_FUSE
 
 @pytest.mark.parametrize("n,cutoff,sched,batch,dist", [
     (512, 256, "B", 1, "uniform"), (512, 256, "B", 1, "int8"),      # the small configuration: 128 CTAs of the small tile
-    (64, 32, "B", 1, "int8"), (2, 1, "B", 3, "int8"), (6, 3, "B", 1, "int8"),
+    (64, 32, "B", 1, "int8"), (2, 1, "B", 3, "int8"), (6, 3, "B", 1, "int8"), (3, 1, "B", 2, "int8"), (7, 3, "B", 1, "int8"),
+    (33, 16, "B", 1, "normal"),
     (100, 50, "B", 2, "normal"),        # ragged tiles in both directions, inner dimension not a multiple of 16
     (101, 50, "B", 2, "int8"),          # odd parent: rank-one term inside the kernel, then the peeled column and row
     (258, 129, "B", 1, "int8"),         # odd quadrant size: 8-byte copies only
