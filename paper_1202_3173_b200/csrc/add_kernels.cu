@@ -427,6 +427,161 @@ __global__ void __launch_bounds__(TX *TY) recombine2_kernel(const Node *__restri
 }
 
 // ---------------------------------------------------------------------------------------
+// The two-level passes for children of ODD size h = 2q + 1 (parent m = 2h, children peeled, grandchildren q).
+// Thread (r, c) with r, c <= q: for r, c < q it owns the 4 x 4 lattice of parent positions whose child-local
+// rows are {r, q + r} and columns {c, q + c} -- exactly the even pass, except that a child's quadrants start at
+// h, not 2q; a thread with r = q (c = q) owns the children's peeled row (column) 2q instead.  Differences from
+// the even pass: the children's sums are written in all four quadrants and on the peeled row and column (their
+// own peeling fix-ups read the whole operands); in the recombination every child's product gets the rank-one
+// term of its peeled split, Acol_j[row] * Brow_j[col], before the parent's U-chain, and the children's last row
+// and column -- thin products written into their Q slots beforehand -- are read from memory by the edge threads.
+// Same operations in the same order per element as one pass per level.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void child_sums(int side, double x11, double x12, double x21, double x22, double (&y)[7], double (&s)[4])
+{
+    if (side == 0) {
+        s[0] = x21 + x22;       // T2
+        s[1] = s[0] - x11;      // T3
+        s[2] = x11 - x21;       // T4
+        s[3] = x12 - s[1];      // T5
+        y[0] = x11; y[1] = x12; y[2] = s[0]; y[3] = s[1]; y[4] = s[2]; y[5] = s[3]; y[6] = x22;
+    } else {
+        s[0] = x12 - x11;       // S2
+        s[1] = x22 - s[0];      // S3
+        s[2] = x22 - x12;       // S4
+        s[3] = s[1] - x21;      // S6
+        y[0] = x11; y[1] = x21; y[2] = s[0]; y[3] = s[1]; y[4] = s[2]; y[5] = x22; y[6] = s[3];
+    }
+}
+
+__global__ void __launch_bounds__(TX *TY) form2_odd_kernel(const Node *__restrict__ parents, Bases bases, Regions2 reg, int q, int item0)
+{
+    const int item = item0 + blockIdx.z;
+    const int par = item >> 1, side = item & 1;
+    const int c = blockIdx.x * TX + threadIdx.x, r = blockIdx.y * TY + threadIdx.y;
+    if (c > q || r > q) return;
+    const int h = 2 * q + 1;
+    const Operand x = side ? parents[par].b : parents[par].a;
+    const double *X = resolve(bases, x);
+    const int64_t ld = x.ld;
+    double *ws = bases.p[BASE_WS];
+    double *child = ws + (side ? reg.child_s : reg.child_t) + int64_t(par) * 4 * reg.child_mat;
+    double *grand = ws + (side ? reg.grand_s : reg.grand_t) + int64_t(par) * 28 * reg.grand_mat;
+    const int64_t cld = reg.child_ld, gld = reg.grand_ld;
+    const int nr = r < q ? 2 : 1, nc = c < q ? 2 : 1;
+    double y[7][2][2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+#pragma unroll
+        for (int v = 0; v < 2; ++v) {
+            if (u >= nr || v >= nc) continue;
+            const int cr = r < q ? u * q + r : 2 * q, cc = c < q ? v * q + c : 2 * q;      // position inside the child
+            const double *p = X + int64_t(cr) * ld + cc;
+            double yy[7], ss[4];
+            child_sums(side, __ldcs(p), __ldcs(p + h), __ldcs(p + int64_t(h) * ld), __ldcs(p + int64_t(h) * ld + h), yy, ss);
+#pragma unroll
+            for (int j = 0; j < 7; ++j) y[j][u][v] = yy[j];
+            const int64_t o = int64_t(cr) * cld + cc;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) child[k * reg.child_mat + o] = ss[k];
+        }
+    if (r >= q || c >= q) return;
+    const int64_t og = int64_t(r) * gld + c;
+#pragma unroll
+    for (int j = 0; j < 7; ++j) {
+        double yy[7], ss[4];
+        child_sums(side, y[j][0][0], y[j][0][1], y[j][1][0], y[j][1][1], yy, ss);
+        double *g = grand + int64_t(j) * 4 * reg.grand_mat + og;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) g[k * reg.grand_mat] = ss[k];
+    }
+}
+
+__device__ __forceinline__ void u_chain7(const double (&k)[7], double &c11, double &c12, double &c21, double &c22)
+{
+    const double u1 = k[0] + k[3], u2 = u1 + k[4], u3 = u1 + k[2];
+    c11 = k[0] + k[1];
+    c12 = u3 + k[5];
+    c21 = u2 - k[6];
+    c22 = u2 + k[2];
+}
+
+__global__ void __launch_bounds__(TX *TY) recombine2_odd_kernel(const Node *__restrict__ parents, const Node *__restrict__ children,
+                                                                Bases bases, Regions2 reg, int q, int item0, int peel)
+{
+    // last parent first: its products are the ones the preceding kernel wrote last, so they are still in L2
+    const int par = item0 + (gridDim.z - 1 - blockIdx.z);
+    const int c = blockIdx.x * TX + threadIdx.x, r = blockIdx.y * TY + threadIdx.y;
+    if (c > q || r > q) return;
+    const int h = 2 * q + 1;
+    const Node *kids = children + size_t(par) * 7;
+    const Operand cc_op = parents[par].c;
+    double *C = resolve(bases, cc_op);
+    const int64_t ldc = cc_op.ld, gld = reg.grand_ld;
+    // peel != 0: the parent itself is odd (size 2h + 1): every entry also gets A[row][2h] * B[2h][col]
+    const double *pacol = nullptr, *pbrow = nullptr;
+    int64_t plda = 0;
+    if (peel) {
+        const Operand pa = parents[par].a, pb = parents[par].b;
+        pacol = resolve(bases, pa) + 2 * h;
+        plda = pa.ld;
+        pbrow = resolve(bases, pb) + int64_t(2 * h) * pb.ld;
+    }
+    auto emit = [&](int cr, int ccol, const double (&z)[7]) {       // the seven child products at child position (cr, ccol)
+        double v[4];
+        u_chain7(z, v[0], v[1], v[2], v[3]);
+#pragma unroll
+        for (int quad = 0; quad < 4; ++quad) {
+            const int R = cr + (quad >> 1) * h, Cc = ccol + (quad & 1) * h;
+            double val = v[quad];
+            if (peel) val = fma(pacol[int64_t(R) * plda], pbrow[Cc], val);
+            C[int64_t(R) * ldc + Cc] = val;
+        }
+    };
+    if (r < q && c < q) {
+        const double *grand = bases.p[BASE_WS] + reg.grand_q + int64_t(par) * 49 * reg.grand_mat + int64_t(r) * gld + c;
+        double z[7][2][2];
+#pragma unroll
+        for (int j = 0; j < 7; ++j) {
+            const double *g = grand + int64_t(j) * 7 * reg.grand_mat;
+            double k[7];
+#pragma unroll
+            for (int t = 0; t < 7; ++t) k[t] = __ldcs(g + t * reg.grand_mat);
+            u_chain7(k, z[j][0][0], z[j][0][1], z[j][1][0], z[j][1][1]);
+            // the rank-one term of child j's own peeled split: its operands' column 2q and row 2q
+            const Operand ka = kids[j].a, kb = kids[j].b;
+            const double *acol = resolve(bases, ka) + 2 * q, *brow = resolve(bases, kb) + int64_t(2 * q) * kb.ld;
+            const double a0 = acol[int64_t(r) * ka.ld], a1 = acol[int64_t(q + r) * ka.ld], b0 = brow[c], b1 = brow[q + c];
+            z[j][0][0] = fma(a0, b0, z[j][0][0]);
+            z[j][0][1] = fma(a0, b1, z[j][0][1]);
+            z[j][1][0] = fma(a1, b0, z[j][1][0]);
+            z[j][1][1] = fma(a1, b1, z[j][1][1]);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+                const double zz[7] = {z[0][u][v], z[1][u][v], z[2][u][v], z[3][u][v], z[4][u][v], z[5][u][v], z[6][u][v]};
+                emit(u * q + r, v * q + c, zz);
+            }
+        return;
+    }
+    // the children's peeled row (r = q) and column (c = q): their products were written by the thin products
+    const int nr = r < q ? 2 : 1, nc = c < q ? 2 : 1;
+    for (int u = 0; u < nr; ++u)
+        for (int v = 0; v < nc; ++v) {
+            const int cr = r < q ? u * q + r : 2 * q, ccol = c < q ? v * q + c : 2 * q;
+            double zz[7];
+#pragma unroll
+            for (int j = 0; j < 7; ++j) {
+                const Operand kc = kids[j].c;
+                zz[j] = resolve(bases, kc)[int64_t(cr) * kc.ld + ccol];
+            }
+            emit(cr, ccol, zz);
+        }
+}
+
+// ---------------------------------------------------------------------------------------
 // Peeling fix-ups for an odd node size m = e + 1 (block algebra on the split
 // A = [A1 ac; ar al], B = [B1 bc; br be]):  the recursion has produced A1.B1 in C[0:e,0:e].
 //   rank-one:    C[r][c] += A[r][e] * B[e][c]            r, c < e
@@ -590,6 +745,8 @@ int launches_of(const Launch &op)
     }
     case OP_FORM2: return chunks(op.count * 2);
     case OP_RECOMBINE2: return chunks(op.count);
+    case OP_FORM2_ODD: return chunks(op.count * 2);
+    case OP_RECOMBINE2_ODD: return chunks(op.count);
     case OP_FORM3: return chunks(op.count * 2);
     case OP_RECOMBINE3: return chunks(op.count);
     case OP_FUSED_STEP: return chunks(op.count);
@@ -693,6 +850,31 @@ cudaError_t launch_recombine2(const Node *tab, const Launch &op, const Bases &ba
     FOR_CHUNKS(total) {
         if (vec) launch_recombine2_as<2>(tile_grid(q, 2, zn), block, stream, tab, op, bases, q, item0);
         else launch_recombine2_as<1>(tile_grid(q, 1, zn), block, stream, tab, op, bases, q, item0);
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_form2_odd(const Node *tab, const Launch &op, const Bases &bases, cudaStream_t stream, int *launched)
+{
+    const dim3 block(TX, TY);
+    const int64_t total = op.count * 2, q = op.h / 2;       // op.h = 2q + 1
+    FOR_CHUNKS(total) {
+        const dim3 grid(unsigned((q + 1 + TX - 1) / TX), unsigned((q + 1 + TY - 1) / TY), unsigned(zn));
+        form2_odd_kernel<<<grid, block, 0, stream>>>(tab + op.parent_tab, bases, op.reg, int(q), int(item0));
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_recombine2_odd(const Node *tab, const Launch &op, const Bases &bases, cudaStream_t stream, int *launched)
+{
+    const dim3 block(TX, TY);
+    const int64_t total = op.count, q = op.h / 2;
+    FOR_CHUNKS(total) {
+        const dim3 grid(unsigned((q + 1 + TX - 1) / TX), unsigned((q + 1 + TY - 1) / TY), unsigned(zn));
+        recombine2_odd_kernel<<<grid, block, 0, stream>>>(tab + op.parent_tab, tab + op.child_tab, bases, op.reg, int(q), int(item0),
+                                                          op.peel_fused);
         ++*launched;
     }
     return cudaGetLastError();

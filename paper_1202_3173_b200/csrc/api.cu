@@ -68,8 +68,8 @@ namespace {
 // Kernel family (strassen_kernel_kind) a launch is counted and timed under.
 int family(int op_kind)
 {
-    if (op_kind == OP_FORM2 || op_kind == OP_FORM3) return STRASSEN_K_FORM;
-    if (op_kind == OP_RECOMBINE2 || op_kind == OP_RECOMBINE3) return STRASSEN_K_RECOMBINE;
+    if (op_kind == OP_FORM2 || op_kind == OP_FORM3 || op_kind == OP_FORM2_ODD) return STRASSEN_K_FORM;
+    if (op_kind == OP_RECOMBINE2 || op_kind == OP_RECOMBINE3 || op_kind == OP_RECOMBINE2_ODD) return STRASSEN_K_RECOMBINE;
     if (op_kind == OP_SCALE_IN || op_kind == OP_SCALE_OUT) return STRASSEN_K_SCALE;
     if (op_kind == OP_FUSED_STEP) return STRASSEN_K_FUSED_STEP;
     if (op_kind == OP_LINCOMB) return STRASSEN_K_LINCOMB;
@@ -204,6 +204,8 @@ int enqueue_launches(strassen_plan *p, const Bases &bases, bool bases16, cudaStr
         case OP_PEEL: e = launch_peel(p->d_tab, op, bases, stream, &launched); break;
         case OP_FORM2: e = launch_form2(p->d_tab, op, bases, vec, stream, &launched); break;
         case OP_RECOMBINE2: e = launch_recombine2(p->d_tab, op, bases, vec, stream, &launched); break;
+        case OP_FORM2_ODD: e = launch_form2_odd(p->d_tab, op, bases, stream, &launched); break;
+        case OP_RECOMBINE2_ODD: e = launch_recombine2_odd(p->d_tab, op, bases, stream, &launched); break;
         case OP_FORM3: e = launch_form3(p->d_tab, op, bases, stream, &launched); break;
         case OP_RECOMBINE3: e = launch_recombine3(p->d_tab, op, bases, stream, &launched); break;
         case OP_LINCOMB: {

@@ -26,6 +26,9 @@ cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bas
 cudaError_t launch_form2(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream, int *launched);
 cudaError_t launch_recombine2(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,
                               int *launched);
+// Two BFS levels in one pass where the children have odd size.
+cudaError_t launch_form2_odd(const Node *tab, const Launch &op, const Bases &bases, cudaStream_t stream, int *launched);
+cudaError_t launch_recombine2_odd(const Node *tab, const Launch &op, const Bases &bases, cudaStream_t stream, int *launched);
 // Items (gridDim.z) one launch of a streaming kernel covers; longer lists are cut into several launches.
 constexpr int kMaxItemsPerLaunch = 32768;
 

@@ -81,10 +81,10 @@ struct Builder {
         const LevelInfo &lv = p->levels.back();
         return fused_step_chosen(p->fused_step, p->schedule, lv.h, lv.parents);
     }
-    int group_size(int level) const
+    int group_size(int level, bool *odd_pair) const
     {
         const std::string sched = fused_last() ? p->schedule.substr(0, p->schedule.size() - 1) : p->schedule;
-        return fused_group_size(p->sizes, sched, level, p->max_fused_levels);
+        return fused_group_size(p->sizes, sched, level, p->max_fused_levels, odd_pair);
     }
 
     // nodes of `level` are p->nodes[tab .. tab + count)
@@ -120,7 +120,8 @@ struct Builder {
             f.kind = OP_FORM; f.level = level; f.j = -1; f.vec_ok = parents_even;
             f.parent_tab = tab; f.child_tab = ctab; f.count = N; f.m = lv.m; f.h = h;
             f.grand_tab = -1;
-            const int group = group_size(level);
+            bool odd_pair = false;
+            const int group = group_size(level, &odd_pair);
             if (group >= 2) {
                 // several BFS levels in one pass: the sums of the intermediate levels are still written
                 // (the operands below are views into them), their products are not
@@ -134,7 +135,22 @@ struct Builder {
                 f.reg.grand_t = lv2.ws_off; f.reg.grand_s = lv2.ws_off + N2 * 4 * lv2.mat_words;
                 f.reg.grand_q = lv2.ws_off + N2 * 8 * lv2.mat_words; f.reg.grand_mat = lv2.mat_words;
                 f.reg.grand_ld = int32_t(lv2.ldw);
-                if (group == 2) {
+                if (group == 2 && odd_pair) {
+                    // children of odd size: their sums are written in full (their own peeling reads them), their last
+                    // row and column come from thin products, everything else as in the even pair
+                    f.kind = OP_FORM2_ODD;
+                    f.vec_ok = 0;
+                    p->launches.push_back(f);
+                    build(level + 2, gtab, N2 * 7);
+                    Launch x{};
+                    x.kind = OP_PEEL; x.level = level + 1; x.j = -1; x.vec_ok = 0; x.peel_fused = 1;
+                    x.parent_tab = ctab; x.child_tab = -1; x.count = N2; x.m = lv2.m; x.h = lv2.h;
+                    p->launches.push_back(x);
+                    Launch r = f;
+                    r.kind = OP_RECOMBINE2_ODD;
+                    r.peel_fused = lv.peel;
+                    p->launches.push_back(r);
+                } else if (group == 2) {
                     f.kind = OP_FORM2;
                     f.vec_ok = parents_even && (lv2.h & 1) == 0;
                     p->launches.push_back(f);
@@ -230,12 +246,24 @@ struct Builder {
 // A run of BFS levels whose lower members are not peeled (their fix-ups need the children's own
 // products) is cut into groups of the largest allowed size from the bottom, where the bytes are;
 // what is left over forms the group at the top of the run.
-int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused)
+int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused, bool *odd_pair)
 {
     const int L = int(sched.size());
+    if (odd_pair) *odd_pair = false;
     if (max_fused <= 1 || level >= L || sched[level] != 'B') return 1;
     int run = 0;
     while (level + run < L && sched[level + run] == 'B' && (run == 0 || (sizes[level + run] & 1) == 0)) ++run;
+    // A BFS level of odd size right below the run cannot be a lower member of an ordinary group, but it can be the
+    // lower member of a pair (the two-level kernels for odd children): the run's last level pairs with it, and the
+    // levels above are grouped among themselves.  The bytes are at the bottom, so the pair is worth more there.
+    const int next = level + run;
+    if (next < L && sched[next] == 'B' && (sizes[next] & 1)) {
+        if (run == 1) {
+            if (odd_pair) *odd_pair = true;
+            return 2;
+        }
+        run -= 1;
+    }
     if (run <= 1) return 1;
     return run % max_fused == 0 ? max_fused : run % max_fused;
 }
@@ -273,7 +301,7 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
             // into C by the recombination pass below (24 h^2 instead of that pass's h^2 of writes) or, where the
             // sub-problem does not end in one, written and folded by a pass of their own (31 h^2)
             const bool folds = level + 1 < LU && upper[level + 1] == 'B' && (sizes[level + 1] & 1) == 0 &&
-                               fused_group_size(sizes, upper, level + 1, 3) == 1;
+                               fused_group_size(sizes, upper, level + 1, 3, nullptr) == 1;
             out.pass_bytes += visits * (24.0 + (folds ? 23.0 : 31.0)) * h * h * 8.0;
             out.launches += (folds ? 5.0 : 12.0) * sequential;
             visits *= 7.0;
@@ -281,8 +309,14 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
             ++level;
             continue;
         }
-        const int g = fused_group_size(sizes, upper, level, 3);
-        const double words = g == 1 ? 27.0 : g == 2 ? 28.0 + 16.25 : 49.0 + 25.5;    // per parent, in h^2 of its children
+        bool odd_pair = false;
+        const int g = fused_group_size(sizes, upper, level, 3, &odd_pair);
+        // per parent, in h^2 of its children (a pair with odd children writes all four quadrants of their sums)
+        const double words = g == 1 ? 27.0 : g == 2 ? (odd_pair ? 30.0 : 28.0) + 16.25 : 49.0 + 25.5;
+        if (odd_pair) {     // the children's own last column and row: thin products over their operands
+            out.pass_bytes += visits * 7.0 * 2.0 * h * h * 8.0;
+            out.launches += 2.0 * sequential;
+        }
         out.pass_bytes += visits * words * h * h * 8.0;
         out.launches += 2.0 * sequential;
         for (int i = 0; i < g; ++i) visits *= 7.0;

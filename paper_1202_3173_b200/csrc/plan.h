@@ -40,6 +40,8 @@ enum OpKind : int32_t {
     OP_FORM3 = 10,     // three BFS levels at once: sums of the children, grandchildren and great-grandchildren
     OP_RECOMBINE3 = 11, // three BFS levels at once: 343 great-grandchild products -> the parent's C
     OP_FUSED_STEP = 12, // a whole BFS step of the deepest level in one kernel: quadrants of A, B -> C
+    OP_FORM2_ODD = 14,      // two BFS levels at once where the children have odd size (peeled)
+    OP_RECOMBINE2_ODD = 15, // ... and their recombination
     OP_LINCOMB = 13     // generic bilinear scheme: one output matrix per parent as a linear combination (j = index of its LinComb)
 };
 
@@ -116,7 +118,8 @@ struct PlanDesc {
 
 // How many levels, starting at `level`, one pass forms and recombines (1 .. max_fused) under schedule
 // `sched` with level sizes `sizes`; 1 for a DFS level.
-int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused);
+int fused_group_size(const std::vector<int64_t> &sizes, const std::string &sched, int level, int max_fused,
+                     bool *odd_pair = nullptr);   // *odd_pair: a pair whose lower member has odd size
 
 // Whether the deepest level (a BFS step over `parents` nodes with children of size h) runs as one fused kernel.
 bool fused_step_chosen(int mode, const std::string &sched, int64_t h, int64_t parents);

@@ -230,6 +230,26 @@ def test_three_level_passes_cover_odd_parents_ragged_tiles_and_stacked_groups(n,
     check_full(n, cutoff, sched, dist, n + 11)          # and the oracle's definition, whole matrix
 
 
+@pytest.mark.parametrize("n,cutoff,sched,batch,dist", [
+    (6, 1, "BB", 2, "int8"),            # children of size 3, grandchildren of size 1
+    (14, 3, "BB", 1, "int8"), (1030, 257, "BB", 1, "uniform"), (1542, 385, "BB", 2, "normal"),
+    (771, 96, "BBB", 1, "uniform"),     # odd parent with odd children: both rank-one terms in one recombination
+    (2060, 128, "BBBB", 1, "int8"),     # 2060 -> 1030 -> 515 (odd) -> 257 (odd) -> 128: pair (1,2), level 3 alone below it
+    (3086, 771, "BB", 1, "uniform"),    # the deepest pair of the n=12345 tree
+    (1034, 129, "DBB", 1, "int8"), (2068, 129, "BDBB", 1, "int8"),
+])
+def test_pair_of_levels_with_odd_children_gives_the_bits_of_single_level_passes(n, cutoff, sched, batch, dist):
+    A, B = inputs.pair(n, dist, n + 13, device="cuda", batch=None if batch == 1 else batch)
+    paired = run_plan(n, cutoff, sched, A, B, batch=batch, flags=UNFUSED)
+    single = run_plan(n, cutoff, sched, A, B, batch=batch, flags=UNFUSED | binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
+    assert torch.equal(paired, single)
+    p, q = Plan(n, cutoff, sched, batch=batch, flags=UNFUSED), Plan(n, cutoff, sched, batch=batch,
+                                                                  flags=UNFUSED | binding.STRASSEN_FLAG_SINGLE_LEVEL_PASSES)
+    assert p.launches_by_kind()["form"] < q.launches_by_kind()["form"]
+    p.close(); q.close()
+    check_full(n, cutoff, sched, dist, n + 13, batch=batch, flags=UNFUSED)
+
+
 def test_batch_with_two_level_passes():
     check_full(256, 64, "BB", "uniform", 121, batch=6)
     check_full(260, 65, "BB", "int8", 122, batch=3)      # odd quarter size: 8-byte accesses

@@ -217,14 +217,23 @@ def test_launch_lists():
     k = p.launches_by_kind()
     assert k["form"] == 2 and k["recombine"] == 2
     p.close()
-    # a peeled level cannot be a lower member of a group (its fix-ups need the children's products)
-    p = Plan(12345, 771, "BBBB")           # sizes 12345, 6172, 3086, 1543 (odd), 771: group (0,1,2), then (3) alone
+    # a level of odd size cannot be a lower member of an ordinary group (its fix-ups need the children's products), but it
+    # can be the lower member of a pair: sizes 12345, 6172, 3086, 1543 (odd), 771 -> pairs (0,1) and (2,3)
+    p = Plan(12345, 771, "BBBB")
+    k = p.launches_by_kind()
+    assert k["form"] == 2 and k["recombine"] == 2 and k["peel"] == 4      # last column + last row at levels 0 and 3
+    p.close()
+    p = Plan(12345, 771, "BBBB", flags=two)
     k = p.launches_by_kind()
     assert k["form"] == 2 and k["recombine"] == 2
     p.close()
-    p = Plan(12345, 771, "BBBB", flags=two)    # pairs: (0), (1,2), (3)
+    p = Plan(12345, 771, "BBBB", flags=single)
     k = p.launches_by_kind()
-    assert k["form"] == 3 and k["recombine"] == 3
+    assert k["form"] == 4 and k["recombine"] == 4 and k["peel"] == 4
+    p.close()
+    p = Plan(12345, 771, "DBBB")           # below the DFS step: level 1 alone (it folds its products into C), pair (2,3)
+    k = p.launches_by_kind()
+    assert k["form"] == 14 and k["recombine"] == 14 and k["accumulate"] == 0 and k["form_one"] == 5
     p.close()
     # a deepest BFS step whose products would leave most SMs idle runs as one fused kernel (no sums, no products in memory)
     p = Plan(512, 256, "B")
