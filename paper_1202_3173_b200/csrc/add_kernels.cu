@@ -622,10 +622,12 @@ __device__ __forceinline__ void dmma_thin(double &d0, double &d1, double a, doub
         : "d"(a), "d"(b));
 }
 
-constexpr int THIN_WARPS = 4, THIN_STEPS = 8;      // warps per CTA; 4-deep steps per loop iteration
+constexpr int THIN_WARPS = 4;      // warps per CTA.  THIN_STEPS = 4-deep steps per loop iteration: 8, or 16 for launches
+                                   // over a few nodes only, whose few warps need more loads in flight each
 
 // Columns [c0, c0 + nc) of C for rows [0, rows), nc <= 8: a warp owns 8 rows.  g = lane / 4, q = lane % 4:
 // the lane feeds A[row g][k + q] and B[k + q][column g] and receives C[row g][columns 2q, 2q + 1].
+template <int THIN_STEPS>
 __global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_kernel(const Node *__restrict__ nodes, Bases bases, int K, int rows,
                                                                     int c0, int nc, int item0)
 {
@@ -666,7 +668,7 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_kernel(const Node *
 
 // Rows [r0, r0 + nr) of C for columns [0, cols), nr <= 8: a warp owns NT adjacent groups of 8 columns.  The lane
 // feeds A[r0 + g][k + q] (zero for g >= nr) and B[k + q][column g of each group].
-template <int NT>
+template <int NT, int THIN_STEPS>
 __global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_kernel(const Node *__restrict__ nodes, Bases bases, int K, int cols,
                                                                     int r0, int nr, int item0)
 {
@@ -923,7 +925,8 @@ cudaError_t launch_thin_cols(const Node *nodes, const Bases &bases, int K, int r
     const int64_t total = count;
     FOR_CHUNKS(total) {
         const dim3 grid((rows + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
-        thin_cols_kernel<<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        if (int64_t(grid.x) * zn < 8 * int64_t(kNominalSMs)) thin_cols_kernel<16><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        else thin_cols_kernel<8><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
         ++*launched;
     }
     return cudaGetLastError();
@@ -938,10 +941,11 @@ cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int c
     FOR_CHUNKS(total) {
         if (two) {
             const dim3 grid((cols + 16 * THIN_WARPS - 1) / (16 * THIN_WARPS), unsigned(zn));
-            thin_rows_kernel<2><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+            thin_rows_kernel<2, 8><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
         } else {
             const dim3 grid((cols + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
-            thin_rows_kernel<1><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+            if (int64_t(grid.x) * zn < 8 * int64_t(kNominalSMs)) thin_rows_kernel<1, 16><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+            else thin_rows_kernel<1, 8><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
         }
         ++*launched;
     }
