@@ -390,16 +390,22 @@ def run_bfs_step(args, rank, world, dev):
     del A, B
     # the workload's top level is the distributed step; the levels below it run on each GPU
     ops = caps.CudaOps(n // 2, dev, cutoff, None if sched == "auto" else sched[1:])
-    state, ex = caps.BfsStepRank(n, rank, ops), caps.TorchDistExchange()
+    state = caps.BfsStepRank(n, rank, ops)
+    if args.bfs_direct:
+        peers = caps.SymmetricPeers(state)
+        step = lambda: caps.bfs_step_direct(state, A_share, B_share, peers)
+    else:
+        ex = caps.TorchDistExchange()
+        step = lambda: caps.bfs_step(state, A_share, B_share, ex)
     stream = torch.cuda.current_stream()
     for _ in range(args.warmup):
-        caps.bfs_step(state, A_share, B_share, ex)
+        step()
     dist.barrier()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        caps.bfs_step(state, A_share, B_share, ex)
+        step()
     e1.record(stream)
     dist.barrier()
     torch.cuda.synchronize()
@@ -409,7 +415,8 @@ def run_bfs_step(args, rank, world, dev):
             "metric": METRIC, "value": 2.0 * n ** 3 / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": {"workload": describe(args.workload), "parallelism": "one BFS step over 7 GPUs (Algorithm 2, k = 1)",
+            "config": {"workload": describe(args.workload), "parallelism": "one BFS step over 7 GPUs (Algorithm 2, k = 1), "
+                                      + ("direct peer stores and loads" if args.bfs_direct else "three NCCL all-to-alls"),
                        "sub_problem": {"n": n // 2, "schedule": ops.plan.schedule, "levels": ops.plan.level_sizes},
                        "message_words": n * n // (4 * caps.P), "all_to_alls_per_step": 3},
             "gpu_launches": args.steps * (ops.plan.launch_count + 2)}), flush=True)
@@ -462,6 +469,9 @@ def main():
                     help="with --gpus 7: time ONE product spread over the seven GPUs as a BFS step of CAPS (Algorithm 2, "
                          "k = 1: local sums, three all-to-alls over NCCL, the n/2 sub-products on the single-GPU path, local "
                          "combine) instead of seven independent replicas")
+    ap.add_argument("--bfs-direct", action="store_true",
+                    help="with --bfs-step: no messages -- the kernels store to and load from the peers' matrices through "
+                         "symmetric-memory peer pointers")
     ap.add_argument("--check-launch", action="store_true",
                     help="no GPU work: every rank joins a gloo group and exchanges a stand-in time through the same reduction "
                          "(checks the launcher plumbing of --gpus N on a machine without GPUs)")

@@ -13,6 +13,13 @@ strassen_dgemm, strassen_bfs_combine_shares); this module only owns buffers and 
   another GPU's memory.
 * `InProcessExchange` delivers the same messages between seven rank objects that live in one process, so the
   whole code path can be checked on a single GPU.
+* The direct form (`bfs_step_direct`, `DirectPeers`) has no messages at all: the formation kernel of rank r stores
+  block r of T_j and S_j straight into rank j's operand matrices, and the combination kernel of rank r loads block r
+  of Q_j straight from rank j's product -- plain stores and loads of the library's own kernels through peer
+  pointers (over NVLink when the ranks are different GPUs), so the transfer is the kernel's own memory traffic and
+  overlaps its arithmetic element by element.  Two barriers per step order writers before readers.  The peer
+  pointers come from `InProcessPeers` (seven ranks of one process: the single-GPU check) or `SymmetricPeers`
+  (torch symmetric memory on a group of seven GPUs; not exercised on hardware in this repository's tests).
 
 Seven ranks take part; on an eight-GPU node one GPU stays idle (the paper itself leaves up to 6/7 of the
 processors idle at P = c 7^k, Section 5.5).
@@ -79,6 +86,22 @@ class CudaOps:
         binding.strassen_bfs_form_shares(rows, self.h, A_share.data_ptr(), A_share.stride(0), B_share.data_ptr(),
                                          B_share.stride(0), [T_send[j].data_ptr() for j in range(P)],
                                          [S_send[j].data_ptr() for j in range(P)], self.h, self._stream())
+
+    def form_into(self, A_share, B_share, T_addresses, S_addresses):
+        """As `form`, the seven blocks of each side going to the given device addresses (rows x h, leading dimension h)."""
+        rows = A_share.shape[0] // 2
+        if rows == 0:
+            return
+        binding.strassen_bfs_form_shares(rows, self.h, A_share.data_ptr(), A_share.stride(0), B_share.data_ptr(),
+                                         B_share.stride(0), T_addresses, S_addresses, self.h, self._stream())
+
+    def combine_from(self, Q_addresses, C_share):
+        """As `combine`, the seven blocks of products read from the given device addresses."""
+        rows = C_share.shape[0] // 2
+        if rows == 0:
+            return
+        binding.strassen_bfs_combine_shares(rows, self.h, Q_addresses, self.h, C_share.data_ptr(), C_share.stride(0),
+                                            self._stream())
 
     def multiply(self, T_full, S_full, Q_full):
         self.plan(T_full, S_full, out=Q_full)
@@ -213,4 +236,93 @@ def bfs_step_in_process(ranks, A, B):
     C = torch.empty_like(A)
     for st in ranks:
         put_share(C, st.combine(), st.rank)
+    return C
+
+
+# ---- the direct form: no messages, the kernels store to and load from the peers' matrices -------------------
+
+class InProcessPeers:
+    """Peer addresses for seven ranks that live in this process (on one device): the operand and product matrices
+    of the BfsStepRank objects themselves.  `barrier` has nothing to wait for: the ranks run one after another on
+    one stream."""
+
+    def __init__(self, ranks):
+        if len(ranks) != P:
+            raise ValueError("seven ranks expected")
+        self.T = [st.T_full.data_ptr() for st in ranks]
+        self.S = [st.S_full.data_ptr() for st in ranks]
+        self.Q = [st.Q_full.data_ptr() for st in ranks]
+
+    def barrier(self):
+        pass
+
+
+class SymmetricPeers:
+    """Peer addresses on a group of seven GPUs: each rank's T, S and Q matrices are allocated in torch symmetric
+    memory, whose rendezvous maps every rank's buffer into every process.  `adopt` replaces the rank's three
+    matrices by views of its own symmetric buffer; `barrier` orders all ranks (and their streams).  This class is
+    glue around torch's symmetric-memory module and is not exercised by the tests here (it needs seven GPUs)."""
+
+    def __init__(self, rank_state, group=None):
+        import torch
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm
+        h = rank_state.h
+        self._dist, self._torch = dist, torch
+        buf = symm.empty(3 * h * h, dtype=torch.float64, device=rank_state.T_full.device)
+        self._handle = symm.rendezvous(buf, group if group is not None else dist.group.WORLD)
+        self._buf = buf
+        bases = [int(p) for p in self._handle.buffer_ptrs]
+        if len(bases) != P:
+            raise ValueError("the BFS step runs on a group of exactly %d ranks" % P)
+        words = h * h * 8
+        self.T = bases
+        self.S = [b + words for b in bases]
+        self.Q = [b + 2 * words for b in bases]
+        rank_state.T_full = buf[:h * h].view(h, h)
+        rank_state.S_full = buf[h * h:2 * h * h].view(h, h)
+        rank_state.Q_full = buf[2 * h * h:].view(h, h)
+
+    def barrier(self):
+        self._torch.cuda.current_stream().synchronize()      # this rank's stores and loads have completed ...
+        self._dist.barrier()                                  # ... and so have every other rank's
+
+
+def form_direct(st: BfsStepRank, A_share, B_share, peers) -> None:
+    """Rank st.rank forms its blocks and stores block `rank` of T_j, S_j into rank j's matrices (rows of rank j's
+    h x h operands that belong to this rank)."""
+    off = st.blocks[st.rank][0] * st.h * 8
+    st.ops.form_into(A_share, B_share, [peers.T[j] + off for j in range(P)], [peers.S[j] + off for j in range(P)])
+
+
+def combine_direct(st: BfsStepRank, peers):
+    """Rank st.rank loads block `rank` of every Q_j from rank j's product and combines them into its share of C."""
+    off = st.blocks[st.rank][0] * st.h * 8
+    st.ops.combine_from([peers.Q[j] + off for j in range(P)], st.C_share)
+    return st.C_share
+
+
+def bfs_step_direct(st: BfsStepRank, A_share, B_share, peers):
+    """The whole step on one rank without messages.  A barrier before the products (all blocks of T_rank, S_rank
+    have been stored by their owners) and one before the combination (all products are complete)."""
+    form_direct(st, A_share, B_share, peers)
+    peers.barrier()
+    st.multiply()
+    peers.barrier()
+    out = combine_direct(st, peers)
+    peers.barrier()          # nobody overwrites its operands or product while a peer may still read or write them
+    return out
+
+
+def bfs_step_direct_in_process(ranks, A, B):
+    """All seven ranks one after another in this process with the direct form: C = A @ B."""
+    import torch
+    peers = InProcessPeers(ranks)
+    for st in ranks:
+        form_direct(st, take_share(A, st.rank), take_share(B, st.rank), peers)
+    for st in ranks:
+        st.multiply()
+    C = torch.empty_like(A)
+    for st in ranks:
+        put_share(C, combine_direct(st, peers), st.rank)
     return C

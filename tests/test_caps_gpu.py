@@ -55,6 +55,28 @@ def test_seven_ranks_in_turn_on_one_gpu_give_the_product(n, cutoff, sched, dist)
         assert all(t.numel() == n * n // (4 * P) for _, _, t in ranks[0].sends_ts() + ranks[0].sends_q())
 
 
+@pytest.mark.parametrize("n,cutoff,sched,dist", [(1400, 350, "B", "uniform"), (1030, 129, "BB", "int8"), (12, 3, "B", "int8")])
+def test_direct_form_without_messages_gives_the_same_bits(n, cutoff, sched, dist):
+    """The formation kernels store straight into the other ranks' operand matrices and the combination kernels load
+    straight from their products (peer addresses; here all seven ranks share one device)."""
+    A, B = inputs.pair(n, dist, 820 + n, device="cuda")
+    dev = A.device
+    def ranks():
+        return [caps.BfsStepRank(n, r, caps.CudaOps(n // 2, dev, cutoff, sched)) for r in range(P)]
+    a, b = ranks(), ranks()
+    C_msg = caps.bfs_step_in_process(a, A, B)
+    C_dir = caps.bfs_step_direct_in_process(b, A, B)
+    torch.cuda.synchronize()
+    assert torch.equal(C_msg, C_dir)
+    for st in a + b:
+        st.ops.close()
+    ref = oracle.classical(A.cpu().numpy(), B.cpu().numpy())
+    if dist == "int8":
+        assert np.array_equal(C_dir.cpu().numpy(), ref)
+    else:
+        assert float(np.abs(C_dir.cpu().numpy() - ref).max()) <= 0.02 * 1e-11 * n * float(A.abs().max()) * float(B.abs().max())
+
+
 def test_share_entry_points_reject_bad_arguments():
     x = torch.zeros(64, dtype=torch.float64, device="cuda")
     seven = [x.data_ptr()] * P
