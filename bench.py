@@ -45,9 +45,10 @@ PER_CONFIG = (("n512", 200), ("n4096", 20), ("b32n2048", 10), ("n12345", 5), ("n
 METRIC = "effective FP64 GFLOP/s (2n^3/t)"
 UNIT = "GFLOP/s"
 
-# DRAM bytes (read + write) of the dominant kernel's launches per step, from one ncu capture of that workload
-# (profiles/gemm_f64_kernel_343x512.md); None where no capture of that exact launch exists.
-GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.125e9, "gemm512x343": 2.125e9}
+# DRAM bytes (read + write) of the dominant kernel's launches per step, from ncu captures of that workload
+# (profiles/launch_list_bench_n4096.md: 1.506 GB read + 0.683 GB written; profiles/gemm_f64_kernel_343x512.md);
+# None where no capture of that exact launch exists.
+GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.19e9, "gemm512x343": 2.125e9}
 
 # FP64 arithmetic peak from unit counts and clocks: 148 SMs x 64 FP64 FMA lanes x 2 flop x 1.965 GHz
 FP64_PEAK_NOMINAL_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
