@@ -57,6 +57,8 @@ template <int BM_, int BN_, int WTM_, int BK_, int STAGES_, int CTAS_> struct Cf
 using CfgWide = Cfg<128, 128, 64, 16, 4, 1>;    // 8 warps of 64 x 32; 149.5 KB of shared memory, one CTA per SM
 using CfgSmall = Cfg<64, 64, 32, 16, 4, 2>;     // 4 warps of 32 x 32; 54 KB: four times as many tiles, for launches
                                                 // whose 128 x 128 tiles would leave most SMs idle
+using CfgTiny = Cfg<32, 64, 16, 16, 4, 3>;      // 4 warps of 16 x 32; 40 KB: eight times as many tiles, for launches whose
+                                                // 64 x 64 tiles would not even fill the two CTA slots of every SM
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
 {
@@ -407,6 +409,8 @@ cudaError_t configure_gemm_kernels()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(gemm_f64_kernel<CfgSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgSmall::SMEM_BYTES));
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemm_f64_kernel<CfgTiny>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgTiny::SMEM_BYTES));
+    if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) g_configured[dev].store(true, std::memory_order_release);
     return cudaSuccess;
 }
@@ -424,8 +428,11 @@ cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, i
         const int nreg = gemm_regions(M, op.count, sm_count, regions);
         for (int i = 0; i < nreg && err == cudaSuccess; ++i) {
             ++*launched;
-            err = regions[i].small ? launch_cfg<CfgSmall>(nodes, bases, regions[i], K, sm_count, stream)
-                                   : launch_cfg<CfgWide>(nodes, bases, regions[i], K, sm_count, stream);
+            const GemmRegion &r = regions[i];
+            const int64_t tiles64 = int64_t((r.row_end - r.row0 + 63) / 64) * ((r.col_end - r.col0 + 63) / 64) * r.leaves;
+            if (!r.small) err = launch_cfg<CfgWide>(nodes, bases, r, K, sm_count, stream);
+            else if (gemm_uses_tiny_tiles(tiles64, sm_count)) err = launch_cfg<CfgTiny>(nodes, bases, r, K, sm_count, stream);
+            else err = launch_cfg<CfgSmall>(nodes, bases, r, K, sm_count, stream);
         }
         if (err != cudaSuccess) return err;
     }

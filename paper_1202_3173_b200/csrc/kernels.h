@@ -145,6 +145,9 @@ struct LinComb;
 cudaError_t launch_lincomb(const Node *tab, const Launch &op, const LinComb &lc, const Bases &bases, bool vec, cudaStream_t stream,
                            int *launched);
 
+// A launch on 64 x 64 tiles that cannot fill the two CTA slots of every SM runs on 32 x 64 tiles instead.
+inline bool gemm_uses_tiny_tiles(int64_t tiles64, int sms) { return tiles64 < 2 * int64_t(sms); }
+
 constexpr int kNominalSMs = 148;   // B200; used where launches are counted without a device at hand
 
 // Sets the shared-memory attribute of every GEMM kernel shape on the current device (idempotent).

@@ -346,9 +346,15 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         for (int i = 0; i < nreg; ++i) {
             const GemmRegion &r = regions[i];
             const int t = r.small ? 64 : 128;
-            const double tiles = double((r.row_end - r.row0 + t - 1) / t) * double((r.col_end - r.col0 + t - 1) / t) * double(r.leaves);
-            const double slots = r.small ? 2.0 * kNominalSMs : double(kNominalSMs);
-            const double tile_us = r.small ? wide_tile_us * 0.5 / 0.88 : wide_tile_us;
+            double slots = r.small ? 2.0 * kNominalSMs : double(kNominalSMs);
+            double tile_us = r.small ? wide_tile_us * 0.5 / 0.88 : wide_tile_us;
+            double tiles = double((r.row_end - r.row0 + t - 1) / t) * double((r.col_end - r.col0 + t - 1) / t) * double(r.leaves);
+            if (r.small && gemm_uses_tiny_tiles(int64_t(tiles / sequential), kNominalSMs)) {
+                // 32 x 64 tiles: twice as many, a fifth of a large tile's time each while an SM holds one or two of them
+                tiles *= 2.0;
+                slots = 1.5 * kNominalSMs;
+                tile_us = wide_tile_us * 0.2;
+            }
             double rounds = tiles / sequential / slots;          // per launch: a DFS level above runs its sub-trees one by one
             if (rounds < 1.0) rounds = 1.0;
             out.product_us += rounds * tile_us * sequential;
