@@ -470,6 +470,8 @@ __global__ void __launch_bounds__(TX *TY) form2_odd_kernel(const Node *__restric
     const int64_t cld = reg.child_ld, gld = reg.grand_ld;
     const int nr = r < q ? 2 : 1, nc = c < q ? 2 : 1;
     double y[7][2][2];
+    // all loads of the thread first (up to 16), then the sums
+    double xv[2][2][4];
 #pragma unroll
     for (int u = 0; u < 2; ++u)
 #pragma unroll
@@ -477,8 +479,19 @@ __global__ void __launch_bounds__(TX *TY) form2_odd_kernel(const Node *__restric
             if (u >= nr || v >= nc) continue;
             const int cr = r < q ? u * q + r : 2 * q, cc = c < q ? v * q + c : 2 * q;      // position inside the child
             const double *p = X + int64_t(cr) * ld + cc;
+            xv[u][v][0] = __ldcs(p);
+            xv[u][v][1] = __ldcs(p + h);
+            xv[u][v][2] = __ldcs(p + int64_t(h) * ld);
+            xv[u][v][3] = __ldcs(p + int64_t(h) * ld + h);
+        }
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+#pragma unroll
+        for (int v = 0; v < 2; ++v) {
+            if (u >= nr || v >= nc) continue;
+            const int cr = r < q ? u * q + r : 2 * q, cc = c < q ? v * q + c : 2 * q;
             double yy[7], ss[4];
-            child_sums(side, __ldcs(p), __ldcs(p + h), __ldcs(p + int64_t(h) * ld), __ldcs(p + int64_t(h) * ld + h), yy, ss);
+            child_sums(side, xv[u][v][0], xv[u][v][1], xv[u][v][2], xv[u][v][3], yy, ss);
 #pragma unroll
             for (int j = 0; j < 7; ++j) y[j][u][v] = yy[j];
             const int64_t o = int64_t(cr) * cld + cc;
