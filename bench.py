@@ -752,9 +752,10 @@ def main():
         "cpu_baseline": cpu,
         "per_config": per_config,
     }
-    print(json.dumps(line), flush=True)
     if world > 1:
-        dist.destroy_process_group()
+        dist.destroy_process_group()         # first: whatever the communicator logs on its way out stays above the line
+    sys.stdout.flush()
+    print(json.dumps(line), flush=True)      # the last line of stdout
 
 
 if __name__ == "__main__":
