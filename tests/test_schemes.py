@@ -25,6 +25,25 @@ WINOGRAD = (2, 7,
 SCHEMES = {"classical": CLASSICAL, "strassen": STRASSEN, "winograd": WINOGRAD}
 
 
+def redundant_classical():
+    """The <2,2,2;8> classical products repeated (12, 8, 4, 4, 9, 9, 9, 9 copies: q = 64) with coefficients that sum to 1 per
+    product (+1 / -1 alternating for an odd count, one coefficient 2 for an even one): a legal scheme whose first block of
+    C adds 20 products -- more than one launch of the linear-combination kernel takes."""
+    n0, q8, u8, v8, w8 = CLASSICAL
+    copies = [12, 8, 4, 4, 9, 9, 9, 9]
+    u, v, w = [], [], [[] for _ in range(4)]
+    for j, n in enumerate(copies):
+        coef = [1 if i % 2 == 0 else -1 for i in range(n)]
+        if n % 2 == 0:
+            coef[0] = 2
+        assert sum(coef) == 1
+        for c in coef:
+            u.append(u8[j]); v.append(v8[j])
+            for b in range(4):
+                w[b].append(c * w8[b][j])
+    return 2, sum(copies), u, v, w
+
+
 def _ints(n, seed):
     rng = np.random.default_rng(seed)
     return rng.integers(-8, 9, (n, n)).astype(float), rng.integers(-8, 9, (n, n)).astype(float)
@@ -33,7 +52,7 @@ def _ints(n, seed):
 # ---- oracle pins ---------------------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("scheme", [CLASSICAL, STRASSEN, WINOGRAD, oracle.classical_scheme(2), oracle.classical_scheme(3),
-                                    oracle.classical_scheme(4)])
+                                    oracle.classical_scheme(4), redundant_classical()])
 def test_tables_satisfy_the_bilinear_identities(scheme):
     assert oracle.brent_residual(*scheme) == 0
     n0, q, u, v, w = scheme
@@ -70,8 +89,11 @@ def test_oracle_recursion_equals_the_definition_on_integers(scheme, n, cutoff, c
 # ---- the library's host side ----------------------------------------------------------------------------------
 
 def test_library_accepts_correct_tables_and_names_the_broken_identity():
-    for s in (CLASSICAL, STRASSEN, WINOGRAD, oracle.classical_scheme(3)):
+    for s in (CLASSICAL, STRASSEN, WINOGRAD, oracle.classical_scheme(3), redundant_classical()):
         binding.strassen_scheme_check(*s)
+    p = Plan(64, 32, "B", scheme=redundant_classical())        # 20, 8, 18, 18 products per block of C: 2 + 1 + 2 + 2 launches
+    assert p.launches_by_kind()["lincomb"] == 7 and p.base_products == 64
+    p.close()
     n0, q, u, v, w = STRASSEN
     bad = [row[:] for row in w]
     bad[3][1] = 1
@@ -137,7 +159,8 @@ def test_built_in_schemes_give_the_product_for_every_schedule(name, n, cutoff):
 @pytest.mark.parametrize("scheme,n,cutoff,sched,batch", [("strassen", 1024, 128, "BBB", 1), ("classical", 1024, 256, "BD", 1),
                                                          (oracle.classical_scheme(3), 729, 81, "BD", 1),
                                                          (oracle.classical_scheme(4), 512, 32, "DB", 2),
-                                                         ("winograd", 1030, 515, "B", 3), ("strassen", 2048, 256, "DBB", 1)])
+                                                         ("winograd", 1030, 515, "B", 3), ("strassen", 2048, 256, "DBB", 1),
+                                                         (redundant_classical(), 256, 64, "BD", 1)])
 def test_schemes_on_float_data_meet_the_bound(scheme, n, cutoff, sched, batch):
     import torch
     from paper_1202_3173_b200 import inputs
