@@ -197,3 +197,22 @@ def test_winograd_table_agrees_with_the_chained_plan_on_integers_and_graph_repla
         torch.cuda.synchronize()
         assert torch.equal(got, want)
     chained.close(); table.close()
+
+
+@pytest.mark.gpu
+def test_scheme_plan_through_the_host_entry_point():
+    import torch
+    from paper_1202_3173_b200 import inputs
+    n = 192
+    A, B = inputs.pair(n, "int8", 77, device="cpu")
+    A, B = A.pin_memory(), B.pin_memory()
+    for flags in (0, binding.STRASSEN_FLAG_HOST_PIPELINE):
+        plan = Plan(n, 24, "BDB", scheme="classical", flags=flags)
+        C = torch.full((n, n), float("nan"), dtype=torch.float64).pin_memory()
+        for _ in range(2):
+            plan.run_host(A, B, C)
+        torch.cuda.synchronize()
+        plan.close()
+        assert np.array_equal(C.numpy(), oracle.classical(A.numpy(), B.numpy()))
+    with pytest.raises(StrassenError):
+        Plan(n, 24, "BDB", scheme="classical", flags=binding.STRASSEN_FLAG_SCALE_OUTSIDE)     # not for generic schemes
