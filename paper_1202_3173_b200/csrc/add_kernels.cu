@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(TX *TY) form_bfs_kernel(const Node *__restrict
 //   U1 = Q0 + Q3   U2 = U1 + Q4   U3 = U1 + Q2
 //   C11 = Q0 + Q1  C12 = U3 + Q5  C21 = U2 - Q6  C22 = U2 + Q2
 // ---------------------------------------------------------------------------------------
-template <int VEC, int RPT, bool FOLD>
+template <int VEC, int RPT, int FOLD>      // FOLD: 0 = write the product, 1 = fold it, 2 = fold it into a parent that needs tolerant accesses
 __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__restrict__ parents,
                                                                const Node *__restrict__ children, Bases bases,
                                                                int h, int item0, int peel, const Node *__restrict__ dfs_parents,
@@ -153,10 +153,10 @@ __global__ void __launch_bounds__(TX *TY) recombine_bfs_kernel(const Node *__res
                     c21 = V::fma1(a1, b0, c21); c22 = V::fma1(a1, b1, c22);
                 }
                 if (FOLD) {
-                    fold_emit<VEC>(ft, r, c, c11);
-                    fold_emit<VEC>(ft, r, c + h, c12);
-                    fold_emit<VEC>(ft, r + h, c, c21);
-                    fold_emit<VEC>(ft, r + h, c + h, c22);
+                    fold_emit<VEC, FOLD == 2>(ft, r, c, c11);
+                    fold_emit<VEC, FOLD == 2>(ft, r, c + h, c12);
+                    fold_emit<VEC, FOLD == 2>(ft, r + h, c, c21);
+                    fold_emit<VEC, FOLD == 2>(ft, r + h, c + h, c22);
                 } else {
                     V::st(o, c11);
                     V::st(o + h, c12);
@@ -801,11 +801,14 @@ void launch_recombine_as(const dim3 &grid, const dim3 &block, cudaStream_t strea
                          int64_t item0)
 {
     const Node *par = tab + op.parent_tab, *kid = tab + op.child_tab;
-    if (op.fold)
-        recombine_bfs_kernel<VEC, RPT, true><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused,
-                                                                        tab + op.fold_tab, op.fold, op.fold_peel);
+    if (op.fold && op.fold_tolerant && VEC == 2)
+        recombine_bfs_kernel<VEC, RPT, 2><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused,
+                                                                     tab + op.fold_tab, op.fold, op.fold_peel);
+    else if (op.fold)
+        recombine_bfs_kernel<VEC, RPT, 1><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused,
+                                                                     tab + op.fold_tab, op.fold, op.fold_peel);
     else
-        recombine_bfs_kernel<VEC, RPT, false><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused, nullptr, 0, 0);
+        recombine_bfs_kernel<VEC, RPT, 0><<<grid, block, 0, stream>>>(par, kid, bases, int(op.h), int(item0), op.peel_fused, nullptr, 0, 0);
 }
 
 cudaError_t launch_recombine(const Node *tab, const Launch &op, const Bases &bases, bool vec, cudaStream_t stream,

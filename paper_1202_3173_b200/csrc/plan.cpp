@@ -102,11 +102,15 @@ struct Builder {
         }
         const LevelInfo &lv = p->levels[level];
         const int64_t h = lv.h, mat = lv.mat_words, ldw = lv.ldw, N = count;
-        bool parents_even = (h & 1) == 0;
+        // 16-byte accesses: what a recombination touches (the parents' C; their A and B only for the rank-one term of an
+        // odd parent) is tracked apart from what a formation touches
+        bool c_even = (h & 1) == 0, ab_even = (h & 1) == 0;
         for (int64_t q = 0; q < N; ++q) {
             const Node &nd = p->nodes[tab + q];
-            parents_even = parents_even && even(nd.a) && even(nd.b) && even(nd.c);
+            c_even = c_even && even(nd.c);
+            ab_even = ab_even && even(nd.a) && even(nd.b);
         }
+        const bool parents_even = c_even && ab_even, recombine_even = c_even && (!lv.peel || ab_even);
         if (lv.mode == 'B' && level == L - 1 && fused_last()) {
             Launch f{};
             f.kind = OP_FUSED_STEP; f.level = level; f.j = -1; f.vec_ok = parents_even;
@@ -158,6 +162,7 @@ struct Builder {
                     Launch r = f;
                     r.kind = OP_RECOMBINE2;
                     r.peel_fused = lv.peel;
+                    r.vec_ok = recombine_even && (lv2.h & 1) == 0;
                     p->launches.push_back(r);
                 } else {
                     const LevelInfo &lv3 = p->levels[level + 2];
@@ -182,6 +187,7 @@ struct Builder {
                 Launch r = f;
                 r.kind = OP_RECOMBINE;
                 r.peel_fused = lv.peel;
+                r.vec_ok = recombine_even;
                 p->launches.push_back(r);
             }
         } else {
@@ -222,7 +228,7 @@ struct Builder {
                     last.fold = j + 1;
                     last.fold_peel = lv.peel && j == 0;
                     last.fold_tab = tab;
-                    last.vec_ok = last.vec_ok && parents_even;
+                    last.fold_tolerant = !recombine_even;      // the sub-problems' own matrices decide last.vec_ok
                     continue;
                 }
                 Launch a = f;

@@ -82,6 +82,8 @@ struct Launch {
                          // products are folded straight into the DFS parents' C quadrants instead of being written (0: no fold)
     int32_t fold_peel;   // ... and the DFS parents have odd size: the first fold (j = 0) carries their rank-one term
     int64_t fold_tab;    // ... index of the first DFS parent node (DFS parent i owns sub-problem node i)
+    int32_t fold_tolerant;   // ... whose C (or B, for the rank-one term) does not allow the 16-byte accesses the sub-problems' own
+                             // matrices allow: the fold checks the alignment of every access to them
     Regions2 reg;        // OP_FORM2 / OP_RECOMBINE2 / OP_FORM3 / OP_RECOMBINE3 only
     Regions3 reg3;       // OP_FORM3 / OP_RECOMBINE3 only
 };
