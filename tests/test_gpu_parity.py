@@ -146,6 +146,48 @@ def test_random_sizes_cutoffs_and_schedules():
         check_full(n, cutoff, sched, "int8", 9000 + case, batch=batch, flags=flags)
 
 
+def test_timed_random_sweep_over_plan_variants():
+    """Random sizes, cutoffs, B/D strings, batches, padded leading dimensions and plan flags (multi-level pass caps, fused
+    step on / off, separate fold passes, graph replay) against the classical oracle, for STRASSEN_FUZZ_SECONDS seconds
+    (default 5; the build's long runs used 300 per seed).  Exact on integer data, within 2 % of the bound on floats."""
+    import os
+    import time
+    budget = float(os.environ.get("STRASSEN_FUZZ_SECONDS", "5"))
+    rng = np.random.default_rng(int(os.environ.get("STRASSEN_FUZZ_SEED", "3")))
+    flag_sets = [0, 1, 32, 64, 128, 256, 64 | 256, 128 | 256, 1 | 128, 32 | 64, 2, 2 | 64]
+    stream = torch.cuda.current_stream().cuda_stream
+    t0, cases = time.time(), 0
+    while time.time() - t0 < budget or cases < 20:
+        n = int(rng.integers(1, 900)) if rng.integers(0, 4) else int(rng.integers(1, 70))
+        cutoff = int(rng.integers(1, max(2, n)))
+        if n // max(cutoff, 1) > 48:
+            cutoff = max(cutoff, n // 48 + 1)
+        L = len(oracle.level_sizes(n, cutoff)) - 1
+        sched = "".join(rng.choice(list("BD"), size=L))
+        flags = int(rng.choice(flag_sets))
+        batch = int(rng.integers(1, 4))
+        pad = int(rng.integers(0, 3)) if batch == 1 else 0
+        dist = "int8" if rng.integers(0, 5) else "uniform"
+        what = (n, cutoff, sched, batch, flags, pad, dist)
+        if pad:
+            ld = n + pad
+            g = torch.Generator("cuda").manual_seed(int(rng.integers(1 << 30)))
+            A = torch.randint(-8, 9, (n, ld), device="cuda", generator=g).double()
+            B = torch.randint(-8, 9, (n, ld), device="cuda", generator=g).double()
+            C = torch.full((n, ld), 7.5, device="cuda", dtype=torch.float64)
+            plan = Plan(n, cutoff, sched, lda=ld, ldb=ld, ldc=ld, flags=flags)
+            ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+            binding.strassen_plan_set_workspace(plan.handle, ws.data_ptr(), plan.workspace_bytes)
+            binding.strassen_dgemm(plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), stream)
+            torch.cuda.synchronize()
+            plan.close()
+            ref = oracle.classical(A[:, :n].cpu().numpy().copy(), B[:, :n].cpu().numpy().copy())
+            assert np.array_equal(C[:, :n].cpu().numpy(), ref) and bool((C[:, n:] == 7.5).all()), what
+        else:
+            check_full(n, cutoff, sched, dist, int(rng.integers(1 << 30)), batch=batch, flags=flags)
+        cases += 1
+
+
 def test_pointers_that_are_only_8_byte_aligned():
     n = 258
     g = torch.Generator("cuda").manual_seed(77)
