@@ -104,6 +104,12 @@ fused_step_kernel(const Node *__restrict__ parents, Bases bases, int h, int item
     const int g = lane >> 2, q = lane & 3;
     const uint32_t smem_base = uint32_t(__cvta_generic_to_shared(smem));
 
+    // Programmatic dependent launch: the launch behind this one in the stream may place its CTAs as soon as
+    // every CTA of this grid has got here, and each grid waits for the whole grid before it (and for its memory)
+    // before its first global access.  A stream of small products then pays the launch and ramp-up of one
+    // product under the tail of the one before.  After any other kind of launch the wait returns at once.
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const Node nd = parents[item0 + blockIdx.z];
     const double *A = base_ptr(bases, nd.a.base) + nd.a.off;
     const double *B = base_ptr(bases, nd.b.base) + nd.b.off;
@@ -367,7 +373,17 @@ template <class F>
 void launch_one(const Node *parents, const Bases &bases, int h, int64_t item0, int64_t zn, int peel, cudaStream_t stream)
 {
     const dim3 grid(unsigned((h + F::TN - 1) / F::TN), unsigned((h + F::TM - 1) / F::TM), unsigned(zn));
-    fused_step_kernel<F><<<grid, F::THREADS, F::SMEM_BYTES, stream>>>(parents, bases, h, int(item0), peel);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(F::THREADS);
+    cfg.dynamicSmemBytes = F::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, fused_step_kernel<F>, parents, bases, h, int(item0), peel);
 }
 
 }  // namespace

@@ -337,7 +337,8 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         const double per_launch = tiles <= kNominalSMs ? slabs * 0.72 : double(int64_t((tiles + 2 * kNominalSMs - 1) / (2 * kNominalSMs))) * slabs * 1.25;
         out.product_us += per_launch * sequential;
         out.product_flops += visits * 7.0 * 2.0 * h * h * h;
-        out.launches += sequential;
+        // launched as a programmatic dependent: its launch and ramp-up run under the tail of the kernel before it
+        out.launches += sequential / 3.0;
         return out;
     }
     const int64_t b = sizes[L];
