@@ -729,6 +729,139 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_kernel(const Node *
     }
 }
 
+// The same thin products for the seven children of one BFS parent at once.  Their large operands are the sums
+// T_0 .. T_6 (S_0 .. S_6) of the parent's four quadrants (Appendix A), so a pass that reads the four quadrants and
+// forms the seven fragments in registers moves 4 h^2 words per parent where seven separate thin products read
+// 7 h^2.  The small operand (the children's own last columns of S_j, last rows of T_j) and the outputs belong to
+// the children: child j of parent p is leaves[7 p + j].  The sums are formed in the order of the formation
+// kernels, so every product sees the values those kernels stored.
+constexpr int SIB_STEPS = 4;       // 4-deep steps per loop iteration: 16 quadrant loads and 28 small loads in flight per lane
+
+// Columns [c0, c0 + nc) of the children's products, all h rows: a warp owns 8 rows of all seven.
+__global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_siblings_kernel(const Node *__restrict__ parents, const Node *__restrict__ leaves,
+                                                                             Bases bases, int h, int c0, int nc, int item0)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
+    const int m0 = (blockIdx.x * THIN_WARPS + warp) * 8;
+    if (m0 >= h) return;
+    const int64_t p = item0 + blockIdx.y;
+    const Node par = parents[p];
+    const Node *kid = leaves + 7 * p;
+    const bool row_ok = m0 + g < h, col_ok = g < nc;
+    const int64_t lda = par.a.ld;
+    const double *x11 = resolve(bases, par.a) + int64_t(row_ok ? m0 + g : 0) * lda + q;
+    const double *x21 = x11 + int64_t(h) * lda;
+    const double *b[7];
+    int64_t ldb[7];
+#pragma unroll
+    for (int j = 0; j < 7; ++j) {
+        const Operand o = kid[j].b;
+        ldb[j] = o.ld;
+        b[j] = resolve(bases, o) + int64_t(q) * o.ld + c0 + (col_ok ? g : 0);
+    }
+    double d[7][2];
+#pragma unroll
+    for (int j = 0; j < 7; ++j) d[j][0] = d[j][1] = 0.0;
+    for (int k0 = 0; k0 < h; k0 += 4 * SIB_STEPS) {
+        double x[SIB_STEPS][4], bv[SIB_STEPS][7];
+        const bool full = k0 + 4 * SIB_STEPS <= h;
+#pragma unroll
+        for (int s = 0; s < SIB_STEPS; ++s) {
+            const int k = k0 + 4 * s;
+            const bool k_ok = full || k + q < h;
+            const bool ok = row_ok && k_ok;
+            x[s][0] = ok ? __ldcs(x11 + k) : 0.0;
+            x[s][1] = ok ? __ldcs(x11 + h + k) : 0.0;
+            x[s][2] = ok ? __ldcs(x21 + k) : 0.0;
+            x[s][3] = ok ? __ldcs(x21 + h + k) : 0.0;
+#pragma unroll
+            for (int j = 0; j < 7; ++j) bv[s][j] = col_ok && k_ok ? b[j][int64_t(k) * ldb[j]] : 0.0;
+        }
+#pragma unroll
+        for (int s = 0; s < SIB_STEPS; ++s) {
+            const double t2 = x[s][2] + x[s][3], t3 = t2 - x[s][0], t4 = x[s][0] - x[s][2], t5 = x[s][1] - t3;
+            dmma_thin(d[0][0], d[0][1], x[s][0], bv[s][0]);
+            dmma_thin(d[1][0], d[1][1], x[s][1], bv[s][1]);
+            dmma_thin(d[2][0], d[2][1], t2, bv[s][2]);
+            dmma_thin(d[3][0], d[3][1], t3, bv[s][3]);
+            dmma_thin(d[4][0], d[4][1], t4, bv[s][4]);
+            dmma_thin(d[5][0], d[5][1], t5, bv[s][5]);
+            dmma_thin(d[6][0], d[6][1], x[s][3], bv[s][6]);
+        }
+    }
+    if (row_ok) {
+#pragma unroll
+        for (int j = 0; j < 7; ++j) {
+            const Operand c = kid[j].c;
+            double *o = resolve(bases, c) + int64_t(m0 + g) * c.ld + c0 + 2 * q;
+            if (2 * q < nc) o[0] = d[j][0];
+            if (2 * q + 1 < nc) o[1] = d[j][1];
+        }
+    }
+}
+
+// Rows [r0, r0 + nr) of the children's products, columns [0, cols): a warp owns 8 columns of all seven.
+__global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_siblings_kernel(const Node *__restrict__ parents, const Node *__restrict__ leaves,
+                                                                             Bases bases, int h, int cols, int r0, int nr, int item0)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
+    const int n0 = (blockIdx.x * THIN_WARPS + warp) * 8;
+    if (n0 >= cols) return;
+    const int64_t p = item0 + blockIdx.y;
+    const Node par = parents[p];
+    const Node *kid = leaves + 7 * p;
+    const bool row_ok = g < nr, col_ok = n0 + g < cols;
+    const int64_t ldb = par.b.ld;
+    const double *y11 = resolve(bases, par.b) + int64_t(q) * ldb + (col_ok ? n0 + g : 0);
+    const double *y21 = y11 + int64_t(h) * ldb;
+    const double *a[7];
+#pragma unroll
+    for (int j = 0; j < 7; ++j) {
+        const Operand o = kid[j].a;
+        a[j] = resolve(bases, o) + int64_t(r0 + (row_ok ? g : 0)) * o.ld + q;
+    }
+    double d[7][2];
+#pragma unroll
+    for (int j = 0; j < 7; ++j) d[j][0] = d[j][1] = 0.0;
+    for (int k0 = 0; k0 < h; k0 += 4 * SIB_STEPS) {
+        double y[SIB_STEPS][4], av[SIB_STEPS][7];
+        const bool full = k0 + 4 * SIB_STEPS <= h;
+#pragma unroll
+        for (int s = 0; s < SIB_STEPS; ++s) {
+            const int k = k0 + 4 * s;
+            const bool k_ok = full || k + q < h;
+            const bool ok = col_ok && k_ok;
+            y[s][0] = ok ? __ldcs(y11 + int64_t(k) * ldb) : 0.0;
+            y[s][1] = ok ? __ldcs(y11 + int64_t(k) * ldb + h) : 0.0;
+            y[s][2] = ok ? __ldcs(y21 + int64_t(k) * ldb) : 0.0;
+            y[s][3] = ok ? __ldcs(y21 + int64_t(k) * ldb + h) : 0.0;
+#pragma unroll
+            for (int j = 0; j < 7; ++j) av[s][j] = row_ok && k_ok ? a[j][k] : 0.0;
+        }
+#pragma unroll
+        for (int s = 0; s < SIB_STEPS; ++s) {
+            const double s2 = y[s][1] - y[s][0], s3 = y[s][3] - s2, s4 = y[s][3] - y[s][1], s6 = s3 - y[s][2];
+            dmma_thin(d[0][0], d[0][1], av[s][0], y[s][0]);
+            dmma_thin(d[1][0], d[1][1], av[s][1], y[s][2]);
+            dmma_thin(d[2][0], d[2][1], av[s][2], s2);
+            dmma_thin(d[3][0], d[3][1], av[s][3], s3);
+            dmma_thin(d[4][0], d[4][1], av[s][4], s4);
+            dmma_thin(d[5][0], d[5][1], av[s][5], y[s][3]);
+            dmma_thin(d[6][0], d[6][1], av[s][6], s6);
+        }
+    }
+    if (row_ok) {
+#pragma unroll
+        for (int j = 0; j < 7; ++j) {
+            const Operand c = kid[j].c;
+            double *o = resolve(bases, c) + int64_t(r0 + g) * c.ld;
+            const int col = n0 + 2 * q;
+            if (col < cols) o[col] = d[j][0];
+            if (col + 1 < cols) o[col + 1] = d[j][1];
+        }
+    }
+}
+
 dim3 tile_grid(int64_t h, int vec, int64_t items)
 {
     return dim3(unsigned((h + TX * vec - 1) / (TX * vec)), unsigned((h + TILE_ROWS - 1) / TILE_ROWS), unsigned(items));
@@ -756,7 +889,7 @@ int launches_of(const Launch &op)
             GemmRegion regions[4];
             tiled = gemm_regions(bulk, op.count, kNominalSMs, regions);
         }
-        return tiled + (rem ? chunks(op.count) * (bulk > 0 ? 2 : 1) : 0);
+        return tiled + (rem ? chunks(gemm_thin_siblings(op) ? op.count / 7 : op.count) * (bulk > 0 ? 2 : 1) : 0);
     }
     case OP_FORM2: return chunks(op.count * 2);
     case OP_RECOMBINE2: return chunks(op.count);
@@ -963,6 +1096,23 @@ cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int c
             if (int64_t(grid.x) * zn < 8 * int64_t(kNominalSMs)) thin_rows_kernel<1, 16><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
             else thin_rows_kernel<1, 8><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
         }
+        ++*launched;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_thin_siblings(const Node *parents, const Node *leaves, const Bases &bases, int h, int M, int rem, int64_t count,
+                                 cudaStream_t stream, int *launched)
+{
+    const int64_t total = count;       // parents; their children are leaves[7 p .. 7 p + 6]
+    FOR_CHUNKS(total) {
+        const dim3 grid((h + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
+        thin_cols_siblings_kernel<<<grid, THIN_WARPS * 32, 0, stream>>>(parents, leaves, bases, h, M, rem, int(item0));
+        ++*launched;
+    }
+    FOR_CHUNKS(total) {
+        const dim3 grid((M + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
+        thin_rows_siblings_kernel<<<grid, THIN_WARPS * 32, 0, stream>>>(parents, leaves, bases, h, M, M, rem, int(item0));
         ++*launched;
     }
     return cudaGetLastError();

@@ -107,7 +107,10 @@ struct LoadState {
     bool interior;          // all rows / columns valid and both operands 16-byte aligned
 };
 
-template <class C>
+// LAST_STEPS: the 4-deep steps of a tile's last 16-deep slab that hold data.  Where K leaves 1..8 columns in
+// it (771 = 48 x 16 + 3: one step) the steps that would multiply zero fill are not issued.  (Taking the short
+// slab first instead, so that the stores still drain beside four steps, measured no gain at all.)
+template <class C, int LAST_STEPS = C::BK / 4>
 __global__ void __launch_bounds__(C::THREADS, C::CTAS)
 gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, GemmRegion reg, int K, int tiles_n, int tiles_per_node, int ktiles,
                 long long total_tiles)
@@ -331,10 +334,10 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, GemmRegion reg, int
             for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
         };
         {
-            double fbL[BK / 4][4], faL[2][BK / 4];
+            double fbL[LAST_STEPS][4], faL[2][LAST_STEPS];
             const double *As = a_frag0 + slot * STAGE_WORDS, *Bs = b_frag0 + slot * STAGE_WORDS;
 #pragma unroll
-            for (int kk = 0; kk < BK / 4; ++kk) {
+            for (int kk = 0; kk < LAST_STEPS; ++kk) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) fbL[kk][j] = Bs[kk * 4 * BS + j * 8];
                 faL[0][kk] = As[kk * 4];
@@ -343,14 +346,14 @@ gemm_f64_kernel(const Node *__restrict__ nodes, Bases bases, GemmRegion reg, int
             for (int i = 0; i < MT; ++i) {
                 if (i + 1 < MT) {
 #pragma unroll
-                    for (int kk = 0; kk < BK / 4; ++kk) faL[(i + 1) & 1][kk] = As[(i + 1) * 8 * AS + kk * 4];
+                    for (int kk = 0; kk < LAST_STEPS; ++kk) faL[(i + 1) & 1][kk] = As[(i + 1) * 8 * AS + kk * 4];
                 } else {
                     cp_async_wait<STAGES - 2>();      // as in slab_steps: the next slab has landed,
                     __syncthreads();                  // and every read of this one has been issued
                     slot = slot + 1 == STAGES ? 0 : slot + 1;
                 }
 #pragma unroll
-                for (int kk = 0; kk < BK / 4; ++kk)
+                for (int kk = 0; kk < LAST_STEPS; ++kk)
 #pragma unroll
                     for (int j = 0; j < 4; ++j) dmma(acc[i][j][0], acc[i][j][1], faL[i & 1][kk], fbL[kk][j]);
                 if (i == 0) issue_load((slot + STAGES - 1) % STAGES);
@@ -377,7 +380,7 @@ cudaError_t configure_gemm_kernels();
 
 namespace {
 
-template <class C>
+template <class C, bool SHORT_OK = false>
 cudaError_t launch_cfg(const Node *nodes, const Bases &bases, const GemmRegion &reg, int K, int sm_count, cudaStream_t stream)
 {
     int dev = 0;
@@ -393,7 +396,14 @@ cudaError_t launch_cfg(const Node *nodes, const Bases &bases, const GemmRegion &
     const long long total = (long long)tiles_per_node * reg.leaves;
     const long long slots = (long long)sm_count * C::CTAS;
     const int grid = int(total < slots ? total : slots);
-    gemm_f64_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(nodes + reg.first, bases, reg, K, tiles_n, tiles_per_node, ktiles, total);
+    const int last_steps = (K - (ktiles - 1) * C::BK + 3) / 4;      // 4-deep steps of the last slab that hold data
+    const Node *first = nodes + reg.first;
+    if (SHORT_OK && last_steps == 1)
+        gemm_f64_kernel<C, SHORT_OK ? 1 : C::BK / 4><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(first, bases, reg, K, tiles_n, tiles_per_node, ktiles, total);
+    else if (SHORT_OK && last_steps == 2)
+        gemm_f64_kernel<C, SHORT_OK ? 2 : C::BK / 4><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(first, bases, reg, K, tiles_n, tiles_per_node, ktiles, total);
+    else
+        gemm_f64_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(first, bases, reg, K, tiles_n, tiles_per_node, ktiles, total);
     return cudaGetLastError();
 }
 
@@ -406,6 +416,10 @@ cudaError_t configure_gemm_kernels()
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && g_configured[dev].load(std::memory_order_acquire)) return cudaSuccess;
     e = cudaFuncSetAttribute(gemm_f64_kernel<CfgWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgWide::SMEM_BYTES));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemm_f64_kernel<CfgWide, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgWide::SMEM_BYTES));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemm_f64_kernel<CfgWide, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgWide::SMEM_BYTES));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(gemm_f64_kernel<CfgSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(CfgSmall::SMEM_BYTES));
     if (e != cudaSuccess) return e;
@@ -430,12 +444,14 @@ cudaError_t launch_gemm(const Node *tab, const Launch &op, const Bases &bases, i
             ++*launched;
             const GemmRegion &r = regions[i];
             const int64_t tiles64 = int64_t((r.row_end - r.row0 + 63) / 64) * ((r.col_end - r.col0 + 63) / 64) * r.leaves;
-            if (!r.small) err = launch_cfg<CfgWide>(nodes, bases, r, K, sm_count, stream);
+            if (!r.small) err = launch_cfg<CfgWide, true>(nodes, bases, r, K, sm_count, stream);
             else if (gemm_uses_tiny_tiles(tiles64, sm_count)) err = launch_cfg<CfgTiny>(nodes, bases, r, K, sm_count, stream);
             else err = launch_cfg<CfgSmall>(nodes, bases, r, K, sm_count, stream);
         }
         if (err != cudaSuccess) return err;
     }
+    if (rem && gemm_thin_siblings(op))
+        return launch_thin_siblings(tab + (op.sibling_tab - 1), nodes, bases, K, M, rem, op.count / 7, stream, launched);
     if (rem) {
         err = launch_thin_cols(nodes, bases, K, K, M, rem, op.count, stream, launched);     // columns [M, K), all rows
         if (err != cudaSuccess) return err;

@@ -49,6 +49,10 @@ cudaError_t launch_thin_cols(const Node *nodes, const Bases &bases, int K, int r
                              cudaStream_t stream, int *launched);
 cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int cols, int r0, int nr, int64_t count,
                              cudaStream_t stream, int *launched);
+// The same for the seven children (size h, leaves[7 p + j]) of each of `count` BFS parents, from the parents' quadrants:
+// columns [M, M + rem) for all rows and rows [M, M + rem) for columns [0, M) of every child's product.
+cudaError_t launch_thin_siblings(const Node *parents, const Node *leaves, const Bases &bases, int h, int M, int rem, int64_t count,
+                                 cudaStream_t stream, int *launched);
 
 // A base product whose size is 1..8 past a multiple of 64 is computed as a tiled bulk of that
 // multiple plus thin products for the remainder rows / columns; returns the remainder (0 = none).
@@ -56,6 +60,12 @@ inline int gemm_thin_remainder(int64_t m)
 {
     const int rem = int(m % 64);
     return rem >= 1 && rem <= 8 ? rem : 0;
+}
+
+// The thin remainders of base products that are whole sets of siblings are computed per parent (from its quadrants).
+inline bool gemm_thin_siblings(const Launch &op)
+{
+    return op.sibling_tab > 0 && op.count % 7 == 0 && gemm_thin_remainder(op.m) != 0 && op.m > 64;
 }
 
 // How the tiled part of a batch of `count` base products with output extent M is launched on a device

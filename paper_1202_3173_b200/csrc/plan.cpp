@@ -87,8 +87,10 @@ struct Builder {
         return fused_group_size(p->sizes, sched, level, p->max_fused_levels, odd_pair);
     }
 
-    // nodes of `level` are p->nodes[tab .. tab + count)
-    void build(int level, int64_t tab, int64_t count)
+    // nodes of `level` are p->nodes[tab .. tab + count); siblings: 1 + the index of their parents' first node where they
+    // are the complete, consecutive sets of seven children of parents whose operands are in memory in full (a BFS step
+    // of its own, or the pair with an odd lower member), 0 otherwise
+    void build(int level, int64_t tab, int64_t count, int64_t siblings = 0)
     {
         if (!err.empty()) return;
         const int L = int(p->levels.size());
@@ -97,6 +99,7 @@ struct Builder {
             g.kind = OP_GEMM; g.level = level; g.j = -1; g.vec_ok = 1;
             g.parent_tab = tab; g.child_tab = -1; g.count = count;
             g.m = p->sizes[level]; g.h = 0;
+            g.sibling_tab = siblings;
             p->launches.push_back(g);
             return;
         }
@@ -145,7 +148,7 @@ struct Builder {
                     f.kind = OP_FORM2_ODD;
                     f.vec_ok = 0;
                     p->launches.push_back(f);
-                    build(level + 2, gtab, N2 * 7);
+                    build(level + 2, gtab, N2 * 7, ctab + 1);
                     Launch x{};
                     x.kind = OP_PEEL; x.level = level + 1; x.j = -1; x.vec_ok = 0; x.peel_fused = 1;
                     x.parent_tab = ctab; x.child_tab = -1; x.count = N2; x.m = lv2.m; x.h = lv2.h;
@@ -158,7 +161,7 @@ struct Builder {
                     f.kind = OP_FORM2;
                     f.vec_ok = parents_even && (lv2.h & 1) == 0;
                     p->launches.push_back(f);
-                    build(level + 2, gtab, N2 * 7);
+                    build(level + 2, gtab, N2 * 7);      // no sibling sets: the pass leaves A21 and B12 of the children's sums unwritten
                     Launch r = f;
                     r.kind = OP_RECOMBINE2;
                     r.peel_fused = lv.peel;
@@ -183,7 +186,7 @@ struct Builder {
                 }
             } else {
                 p->launches.push_back(f);
-                build(level + 1, ctab, N * 7);
+                build(level + 1, ctab, N * 7, tab + 1);
                 Launch r = f;
                 r.kind = OP_RECOMBINE;
                 r.peel_fused = lv.peel;
@@ -295,6 +298,7 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
     }());
     const std::string upper = fused ? sched.substr(0, size_t(L) - 1) : sched;    // levels handled by streaming passes
     const int LU = int(upper.size());
+    bool sibling_leaves = false;      // the base products are whole sets of children of parents that are in memory in full
     for (int level = 0; level < L;) {
         const double m = double(sizes[level]), h = double(sizes[level + 1]);
         if (sizes[level] & 1) {
@@ -313,10 +317,12 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
             visits *= 7.0;
             sequential *= 7.0;
             ++level;
+            sibling_leaves = false;
             continue;
         }
         bool odd_pair = false;
         const int g = fused_group_size(sizes, upper, level, 3, &odd_pair);
+        sibling_leaves = g == 1 || odd_pair;
         // per parent, in h^2 of its children (a pair with odd children writes all four quadrants of their sums)
         const double words = g == 1 ? 27.0 : g == 2 ? (odd_pair ? 30.0 : 28.0) + 16.25 : 49.0 + 25.5;
         if (odd_pair) {     // the children's own last column and row: thin products over their operands
@@ -369,7 +375,8 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         }
     }
     if (rem) {
-        out.thin_bytes += leaves * 2.0 * double(b) * double(b) * 8.0;
+        // one operand of every leaf read in full for each of the two strips, or the four quadrants of the parent for seven leaves
+        out.thin_bytes += leaves * 2.0 * double(b) * double(b) * 8.0 * (sibling_leaves && b > 64 ? 4.0 / 7.0 : 1.0);
         out.launches += 2.0 * sequential;
     }
     return out;

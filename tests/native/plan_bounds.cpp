@@ -45,6 +45,18 @@ static bool check(const PlanDesc &d)
                 return false;
             }
         }
+        if (op.sibling_tab > 0) {       // the leaves are the sevens of children of these parents, whose quadrants the thin products read
+            if (op.count % 7 != 0 || op.sibling_tab - 1 + op.count / 7 > int64_t(d.nodes.size()) || op.sibling_tab - 1 + op.count / 7 > op.parent_tab) {
+                printf("FAIL n=%lld sched=%s: sibling parents out of the node table\n", (long long)d.n, d.schedule.c_str());
+                return false;
+            }
+            for (int64_t i = 0; i < op.count / 7; ++i) {
+                const Node &par = d.nodes[size_t(op.sibling_tab - 1 + i)];
+                if (!inside(par.a, 2 * op.m, 2 * op.m, lim[par.a.base], "sibling parent A", d) ||
+                    !inside(par.b, 2 * op.m, 2 * op.m, lim[par.b.base], "sibling parent B", d))
+                    return false;
+            }
+        }
         // products of one launch must not overlap each other
         std::vector<std::pair<int64_t, int64_t>> spans;
         for (int64_t i = 0; i < op.count; ++i) {

@@ -37,6 +37,21 @@ def test_base_product_thin_remainders(n):
     check_full(n, n, "", "normal", 301 + n, batch=3)
 
 
+@pytest.mark.parametrize("n,cutoff,sched,batch", [(262, 131, "B", 1), (1542, 771, "B", 2), (393, 196, "B", 1), (526, 131, "BB", 3),
+                                                  (1050, 131, "BBB", 1), (524, 131, "BB", 1), (1048, 131, "BBB", 2), (525, 131, "DB", 1)])
+def test_thin_remainders_of_sibling_base_products(n, cutoff, sched, batch):
+    """Base products that are the seven children of BFS parents get their remainder rows and columns per parent, from
+    the parent's quadrants: after a BFS step of its own (262, 1542, odd parent 393, below a DFS step 525) and after the
+    pair with an odd lower member (526: 263 odd).  The even two- and three-level passes (524, 1048) leave one
+    quadrant of the intermediate sums unwritten, so their leaves keep the per-leaf products.  Three-launch path."""
+    no_fused_step = 128
+    p = Plan(n, cutoff, sched, batch=batch, flags=no_fused_step)
+    assert p.launches_by_kind()["gemm"] >= 3          # tiled bulk + two thin launches
+    p.close()
+    check_full(n, cutoff, sched, "int8", 330 + n, batch=batch, flags=no_fused_step)
+    check_full(n, cutoff, sched, "uniform", 331 + n, batch=batch, flags=no_fused_step)
+
+
 @pytest.mark.parametrize("n,cutoff,sched,batch", [(4480, 560, "BBB", 1), (2400, 300, "BBB", 2), (4481, 560, "BBB", 1)])
 def test_base_product_margin_strips(n, cutoff, sched, batch):
     # a base size 1..64 past a multiple of 128 with hundreds of leaves: 128 x 128 tiles over the multiple, a right
