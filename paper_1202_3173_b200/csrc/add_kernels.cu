@@ -640,13 +640,16 @@ constexpr int THIN_WARPS = 4;      // warps per CTA.  THIN_STEPS = 4-deep steps 
 
 // Columns [c0, c0 + nc) of C for rows [0, rows), nc <= 8: a warp owns 8 rows.  g = lane / 4, q = lane % 4:
 // the lane feeds A[row g][k + q] and B[k + q][column g] and receives C[row g][columns 2q, 2q + 1].
-template <int THIN_STEPS>
+// KSPLIT (launches over one or two nodes, which would leave each SM a handful of warps): the CTA owns 8 rows, its
+// warps take the chunks of the inner dimension in turn and warp 0 adds their sums in warp order.
+template <int THIN_STEPS, bool KSPLIT = false>
 __global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_kernel(const Node *__restrict__ nodes, Bases bases, int K, int rows,
                                                                     int c0, int nc, int item0)
 {
+    __shared__ double part[KSPLIT ? THIN_WARPS - 1 : 1][2][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
-    const int m0 = (blockIdx.x * THIN_WARPS + warp) * 8;
-    if (m0 >= rows) return;
+    const int m0 = KSPLIT ? blockIdx.x * 8 : (blockIdx.x * THIN_WARPS + warp) * 8;
+    if (!KSPLIT && m0 >= rows) return;
     const Node nd = nodes[item0 + blockIdx.y];
     const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
     const bool row_ok = m0 + g < rows, col_ok = g < nc;
@@ -654,7 +657,7 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_kernel(const Node *
     const double *b = B + int64_t(q) * nd.b.ld + c0 + (col_ok ? g : 0);
     const int64_t ldb = nd.b.ld;
     double d0 = 0.0, d1 = 0.0;
-    for (int k0 = 0; k0 < K; k0 += 4 * THIN_STEPS) {
+    for (int k0 = KSPLIT ? warp * 4 * THIN_STEPS : 0; k0 < K; k0 += (KSPLIT ? THIN_WARPS : 1) * 4 * THIN_STEPS) {
         double av[THIN_STEPS], bv[THIN_STEPS];
         if (k0 + 4 * THIN_STEPS <= K) {
 #pragma unroll
@@ -672,6 +675,19 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_kernel(const Node *
 #pragma unroll
         for (int s = 0; s < THIN_STEPS; ++s) dmma_thin(d0, d1, av[s], bv[s]);
     }
+    if (KSPLIT) {
+        if (warp > 0) {
+            part[warp - 1][0][lane] = d0;
+            part[warp - 1][1][lane] = d1;
+        }
+        __syncthreads();
+        if (warp > 0) return;
+#pragma unroll
+        for (int w = 0; w < THIN_WARPS - 1; ++w) {
+            d0 += part[w][0][lane];
+            d1 += part[w][1][lane];
+        }
+    }
     if (row_ok) {
         double *o = resolve(bases, nd.c) + int64_t(m0 + g) * nd.c.ld + c0 + 2 * q;
         if (2 * q < nc) o[0] = d0;
@@ -681,13 +697,14 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_kernel(const Node *
 
 // Rows [r0, r0 + nr) of C for columns [0, cols), nr <= 8: a warp owns NT adjacent groups of 8 columns.  The lane
 // feeds A[r0 + g][k + q] (zero for g >= nr) and B[k + q][column g of each group].
-template <int NT, int THIN_STEPS>
+template <int NT, int THIN_STEPS, bool KSPLIT = false>
 __global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_kernel(const Node *__restrict__ nodes, Bases bases, int K, int cols,
                                                                     int r0, int nr, int item0)
 {
+    __shared__ double part[KSPLIT ? THIN_WARPS - 1 : 1][2 * NT][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
-    const int n0 = (blockIdx.x * THIN_WARPS + warp) * 8 * NT;
-    if (n0 >= cols) return;
+    const int n0 = KSPLIT ? blockIdx.x * 8 * NT : (blockIdx.x * THIN_WARPS + warp) * 8 * NT;
+    if (!KSPLIT && n0 >= cols) return;
     const Node nd = nodes[item0 + blockIdx.y];
     const double *A = resolve(bases, nd.a), *B = resolve(bases, nd.b);
     const bool row_ok = g < nr;
@@ -703,7 +720,7 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_kernel(const Node *
     double d[NT][2];
 #pragma unroll
     for (int j = 0; j < NT; ++j) d[j][0] = d[j][1] = 0.0;
-    for (int k0 = 0; k0 < K; k0 += 4 * THIN_STEPS) {
+    for (int k0 = KSPLIT ? warp * 4 * THIN_STEPS : 0; k0 < K; k0 += (KSPLIT ? THIN_WARPS : 1) * 4 * THIN_STEPS) {
         double av[THIN_STEPS], bv[THIN_STEPS][NT];
         const bool full = k0 + 4 * THIN_STEPS <= K;
 #pragma unroll
@@ -717,6 +734,24 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_kernel(const Node *
         for (int s = 0; s < THIN_STEPS; ++s)
 #pragma unroll
             for (int j = 0; j < NT; ++j) dmma_thin(d[j][0], d[j][1], av[s], bv[s][j]);
+    }
+    if (KSPLIT) {
+        if (warp > 0) {
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                part[warp - 1][2 * j][lane] = d[j][0];
+                part[warp - 1][2 * j + 1][lane] = d[j][1];
+            }
+        }
+        __syncthreads();
+        if (warp > 0) return;
+#pragma unroll
+        for (int w = 0; w < THIN_WARPS - 1; ++w)
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                d[j][0] += part[w][2 * j][lane];
+                d[j][1] += part[w][2 * j + 1][lane];
+            }
     }
     if (row_ok) {
         double *o = resolve(bases, nd.c) + int64_t(r0 + g) * nd.c.ld;
@@ -735,9 +770,19 @@ __global__ void __launch_bounds__(THIN_WARPS * 32) thin_rows_kernel(const Node *
 // 7 h^2.  The small operand (the children's own last columns of S_j, last rows of T_j) and the outputs belong to
 // the children: child j of parent p is leaves[7 p + j].  The sums are formed in the order of the formation
 // kernels, so every product sees the values those kernels stored.
-constexpr int SIB_STEPS = 4;       // 4-deep steps per loop iteration: 16 quadrant loads and 28 small loads in flight per lane
+constexpr int SIB_STEPS = 4;       // 4-deep steps per loop iteration: 16 quadrant loads and 28 small loads in flight per lane.
+// The two kernels run at 3.6 and 4.4 TB/s, bound by the latency of those loads at 12 to 16 warps per SM.  Measured and not
+// kept (n = 12345; leaves' remainders + peeled level 3 = 5.8 ms per product as is): 8 steps in registers (peel 3.0 -> 5.1 ms);
+// the seven small vectors of a peeled level staged in shared memory (6.1 ms); the quadrant streams through a per-warp
+// ring of 8-byte cp.async copies, three chunks in flight (peel 4.2 ms, remainders +0.8 ms: 8-byte asynchronous copies are
+// slower than plain loads); the inner dimension split over the warps of a CTA (peel 2.9 ms, remainders +0.2 ms, and a
+// summation order of its own); the small operand loaded once per CTA and chunk by all threads together and handed over through
+// shared memory, one barrier per chunk (peel 3.1 ms, remainders +0.4 ms); 96 or 128 registers for more warps per SM, and plain
+// instead of streaming loads (no gain).  Counters at 49 parents of 771: DRAM 47 %, L2 44 %, L1 data pipe 56 %, DMMA 38 %,
+// 10.7 warps active per SM, long-scoreboard stalls: no unit is saturated, the loop waits on its loads.
 
-// Columns [c0, c0 + nc) of the children's products, all h rows: a warp owns 8 rows of all seven.
+// Columns [c0, c0 + nc) of the children's products, all h rows: a warp owns 8 rows of all seven.  Summation over k ascending,
+// like the per-leaf kernels: plans that differ only in which of the two serves a node give the same bits.
 __global__ void __launch_bounds__(THIN_WARPS * 32) thin_cols_siblings_kernel(const Node *__restrict__ parents, const Node *__restrict__ leaves,
                                                                              Bases bases, int h, int c0, int nc, int item0)
 {
@@ -881,7 +926,8 @@ int launches_of(const Launch &op)
     case OP_RECOMBINE: return chunks(op.count);
     case OP_FORM_ONE: return chunks(op.count * ((op.j >= 2 && op.j <= 4) ? 2 : 1));
     case OP_ACCUMULATE: return chunks(op.count);
-    case OP_PEEL: return (op.peel_fused ? 2 : 3) * chunks(op.count);
+    case OP_PEEL:
+        return (op.peel_fused ? 0 : chunks(op.count)) + 2 * chunks(op.sibling_tab > 0 && op.count % 7 == 0 ? op.count / 7 : op.count);
     case OP_GEMM: {
         const int rem = gemm_thin_remainder(op.m), bulk = int(op.m) - rem;
         int tiled = 0;
@@ -1074,7 +1120,9 @@ cudaError_t launch_thin_cols(const Node *nodes, const Bases &bases, int K, int r
     const int64_t total = count;
     FOR_CHUNKS(total) {
         const dim3 grid((rows + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
-        if (int64_t(grid.x) * zn < 8 * int64_t(kNominalSMs)) thin_cols_kernel<16><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        if (int64_t(grid.x) * zn < 4 * int64_t(kNominalSMs) && K >= 4096)
+            thin_cols_kernel<8, true><<<dim3((rows + 7) / 8, unsigned(zn)), THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
+        else if (int64_t(grid.x) * zn < 8 * int64_t(kNominalSMs)) thin_cols_kernel<16><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
         else thin_cols_kernel<8><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, rows, c0, nc, int(item0));
         ++*launched;
     }
@@ -1093,7 +1141,9 @@ cudaError_t launch_thin_rows(const Node *nodes, const Bases &bases, int K, int c
             thin_rows_kernel<2, 8><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
         } else {
             const dim3 grid((cols + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
-            if (int64_t(grid.x) * zn < 8 * int64_t(kNominalSMs)) thin_rows_kernel<1, 16><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+            if (int64_t(grid.x) * zn < 4 * int64_t(kNominalSMs) && K >= 4096)
+                thin_rows_kernel<1, 8, true><<<dim3((cols + 7) / 8, unsigned(zn)), THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
+            else if (int64_t(grid.x) * zn < 8 * int64_t(kNominalSMs)) thin_rows_kernel<1, 16><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
             else thin_rows_kernel<1, 8><<<grid, THIN_WARPS * 32, 0, stream>>>(nodes, bases, K, cols, r0, nr, int(item0));
         }
         ++*launched;
@@ -1110,7 +1160,7 @@ cudaError_t launch_thin_siblings(const Node *parents, const Node *leaves, const 
         thin_cols_siblings_kernel<<<grid, THIN_WARPS * 32, 0, stream>>>(parents, leaves, bases, h, M, rem, int(item0));
         ++*launched;
     }
-    FOR_CHUNKS(total) {
+    if (M > 0) FOR_CHUNKS(total) {
         const dim3 grid((M + 8 * THIN_WARPS - 1) / (8 * THIN_WARPS), unsigned(zn));
         thin_rows_siblings_kernel<<<grid, THIN_WARPS * 32, 0, stream>>>(parents, leaves, bases, h, M, M, rem, int(item0));
         ++*launched;
@@ -1130,6 +1180,8 @@ cudaError_t launch_peel(const Node *tab, const Launch &op, const Bases &bases, c
             ++*launched;
         }
     }
+    if (op.sibling_tab > 0 && op.count % 7 == 0)      // seven siblings at a time, from their parent's quadrants
+        return launch_thin_siblings(tab + (op.sibling_tab - 1), nodes, bases, m, e, 1, op.count / 7, stream, launched);
     cudaError_t err = launch_thin_cols(nodes, bases, m, m, e, 1, op.count, stream, launched);   // last column, all rows
     if (err != cudaSuccess) return err;
     return launch_thin_rows(nodes, bases, m, e, e, 1, op.count, stream, launched);              // last row, other columns

@@ -152,6 +152,7 @@ struct Builder {
                     Launch x{};
                     x.kind = OP_PEEL; x.level = level + 1; x.j = -1; x.vec_ok = 0; x.peel_fused = 1;
                     x.parent_tab = ctab; x.child_tab = -1; x.count = N2; x.m = lv2.m; x.h = lv2.h;
+                    x.sibling_tab = tab + 1;
                     p->launches.push_back(x);
                     Launch r = f;
                     r.kind = OP_RECOMBINE2_ODD;
@@ -245,6 +246,7 @@ struct Builder {
             Launch x{};
             x.kind = OP_PEEL; x.level = level; x.j = -1; x.vec_ok = 0; x.peel_fused = 1;
             x.parent_tab = tab; x.child_tab = -1; x.count = N; x.m = lv.m; x.h = h;
+            x.sibling_tab = siblings;
             p->launches.push_back(x);
         }
     }
@@ -298,11 +300,12 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
     }());
     const std::string upper = fused ? sched.substr(0, size_t(L) - 1) : sched;    // levels handled by streaming passes
     const int LU = int(upper.size());
-    bool sibling_leaves = false;      // the base products are whole sets of children of parents that are in memory in full
+    bool sibling_leaves = false;      // the nodes of the level at hand are whole sets of children of parents that are in memory in full
     for (int level = 0; level < L;) {
         const double m = double(sizes[level]), h = double(sizes[level + 1]);
         if (sizes[level] & 1) {
-            out.pass_bytes += visits * 2.0 * m * m * 8.0;      // last column and last row: each reads one operand in full
+            // last column and last row: each reads one operand in full, or the parent's four quadrants for seven siblings
+            out.pass_bytes += visits * 2.0 * m * m * 8.0 * (sibling_leaves ? 4.0 / 7.0 : 1.0);
             out.launches += 2.0 * sequential;
         }
         if (level >= LU) break;                                // the fused deepest step: accounted with the products
@@ -326,7 +329,7 @@ ModelParts plan_model_parts(const std::vector<int64_t> &sizes, const std::string
         // per parent, in h^2 of its children (a pair with odd children writes all four quadrants of their sums)
         const double words = g == 1 ? 27.0 : g == 2 ? (odd_pair ? 30.0 : 28.0) + 16.25 : 49.0 + 25.5;
         if (odd_pair) {     // the children's own last column and row: thin products over their operands
-            out.pass_bytes += visits * 7.0 * 2.0 * h * h * 8.0;
+            out.pass_bytes += visits * 4.0 * 2.0 * h * h * 8.0;     // seven siblings from their parent's four quadrants
             out.launches += 2.0 * sequential;
         }
         out.pass_bytes += visits * words * h * h * 8.0;

@@ -84,10 +84,10 @@ struct Launch {
     int64_t fold_tab;    // ... index of the first DFS parent node (DFS parent i owns sub-problem node i)
     int32_t fold_tolerant;   // ... whose C (or B, for the rank-one term) does not allow the 16-byte accesses the sub-problems' own
                              // matrices allow: the fold checks the alignment of every access to them
-    int64_t sibling_tab; // OP_GEMM whose leaves are the complete sets of seven children of the nodes of a BFS step, child j of
-                         // parent i at leaf 7 i + j, and those parents' operands are in memory in full (the even multi-level
+    int64_t sibling_tab; // OP_GEMM / OP_PEEL whose nodes are the complete sets of seven children of the nodes of a BFS step, child j
+                         // of parent i at node 7 i + j, and those parents' operands are in memory in full (the even multi-level
                          // passes skip one quadrant of the intermediate sums): 1 + index of the first of those parents
-                         // (0: none); lets the thin remainders of all seven be computed from the parents' quadrants
+                         // (0: none); lets the thin products of all seven be computed from the parents' quadrants
     Regions2 reg;        // OP_FORM2 / OP_RECOMBINE2 / OP_FORM3 / OP_RECOMBINE3 only
     Regions3 reg3;       // OP_FORM3 / OP_RECOMBINE3 only
 };
