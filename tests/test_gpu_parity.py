@@ -52,6 +52,15 @@ def test_thin_remainders_of_sibling_base_products(n, cutoff, sched, batch):
     check_full(n, cutoff, sched, "uniform", 331 + n, batch=batch, flags=no_fused_step)
 
 
+@pytest.mark.parametrize("n,cutoff,sched", [(4100, 4100, ""), (8197, 4100, "B")])
+def test_thin_products_over_one_large_node(n, cutoff, sched):
+    """A single node with an inner dimension of 4096 or more: its thin products give each CTA 8 rows (columns) and split
+    the inner dimension over the CTA's warps.  4100 = 64 x 64 + 4: remainder columns and rows of one base product;
+    8197: the peeled last column and row of the root (its children, 4098 = 64 x 64 + 2, are one set of siblings)."""
+    check_sampled(n, cutoff, sched, "int8", 350 + n)
+    check_sampled(n, cutoff, sched, "uniform", 351 + n)
+
+
 @pytest.mark.parametrize("n,cutoff,sched,batch", [(4480, 560, "BBB", 1), (2400, 300, "BBB", 2), (4481, 560, "BBB", 1)])
 def test_base_product_margin_strips(n, cutoff, sched, batch):
     # a base size 1..64 past a multiple of 128 with hundreds of leaves: 128 x 128 tiles over the multiple, a right
