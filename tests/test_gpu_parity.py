@@ -356,6 +356,38 @@ def test_fused_step_agrees_with_the_three_launch_path(n, cutoff, sched, batch, d
         check_sampled(n, cutoff, sched, dist, 40 + n, batch=batch, flags=FUSED)
 
 
+def test_fused_step_launched_as_a_dependent_keeps_stream_order():
+    """The fused step is launched with programmatic stream serialisation: its CTAs may be placed while the launch
+    before it still runs, but every global access waits for that launch.  Inputs rewritten by other kernels between
+    products, outputs overwritten by the next product, and a consumer kernel behind each product must all see
+    stream order."""
+    n, steps = 512, 24
+    g = torch.Generator("cuda").manual_seed(5)
+    A = torch.randint(-3, 4, (n, n), device="cuda", generator=g).double()
+    B = torch.randint(-3, 4, (n, n), device="cuda", generator=g).double()
+    A0, B0 = A.cpu().numpy().copy(), B.cpu().numpy().copy()
+    plan = Plan(n, 256, "B", flags=FUSED)
+    assert plan.launches_by_kind() == {**{k: 0 for k in plan.launches_by_kind()}, "fused_step": 1}
+    C = torch.empty_like(A)
+    sums = torch.zeros(steps, dtype=torch.float64, device="cuda")
+    kept = []
+    for i in range(steps):
+        A.add_(1.0)                      # another kernel rewrites an input right before the product ...
+        plan(A, B, out=C)                # ... the product overwrites the output of the one before it ...
+        sums[i] = C.sum()                # ... and a consumer reads it right behind
+        if i % 8 == 7:
+            kept.append((i, C.clone()))
+        B.sub_(1.0)                      # and the other input changes before the next product
+    torch.cuda.synchronize()
+    plan.close()
+    for i in range(steps):
+        ref = oracle.classical(A0 + (i + 1), B0 - i)
+        assert float(sums[i]) == float(ref.sum()), i
+        for k, c in kept:
+            if k == i:
+                assert np.array_equal(c.cpu().numpy(), ref), i
+
+
 def test_fused_step_on_pointers_that_are_only_8_byte_aligned_and_strided_views():
     n, ld = 130, 137
     g = torch.Generator("cuda").manual_seed(9)
