@@ -46,9 +46,9 @@ METRIC = "effective FP64 GFLOP/s (2n^3/t)"
 UNIT = "GFLOP/s"
 
 # DRAM bytes (read + write) of the dominant kernel's launches per step, from ncu captures of that workload
-# (profiles/launch_list_bench_n4096.md: 1.506 GB read + 0.683 GB written; profiles/gemm_f64_kernel_343x512.md);
+# (profiles/launch_list_bench_n4096.md: 1.446 GB read + 0.682 GB written; profiles/gemm_f64_kernel_343x512.md);
 # None where no capture of that exact launch exists.
-GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.19e9, "gemm512x343": 2.125e9}
+GEMM_DRAM_TRAFFIC_BYTES = {"n4096": 2.13e9, "gemm512x343": 2.125e9}
 
 # FP64 arithmetic peak from unit counts and clocks: 148 SMs x 64 FP64 FMA lanes x 2 flop x 1.965 GHz
 FP64_PEAK_NOMINAL_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
@@ -736,7 +736,7 @@ def main():
                      "launches_per_step": head["launches_by_kind"].get(product_kind),
                      "launches": "the family's launches of one step are timed together (two CUDA events around each, a separate "
                                  "pass from the timed region); at n=4096 they are 342 leaves on 128 x 128 tiles and 1 leaf on "
-                                 "64 x 64 tiles",
+                                 "32 x 64 tiles",
                      "traffic": GEMM_DRAM_TRAFFIC_BYTES.get(args.workload),
                      "traffic_source": "one ncu capture of this launch (profiles/), per step; not measured in this run"
                                        if GEMM_DRAM_TRAFFIC_BYTES.get(args.workload) else None},
